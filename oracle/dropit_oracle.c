@@ -1,0 +1,298 @@
+/*
+ * DropIT oracle: a plain, slow, single-file CPU statement of what the DropIT
+ * layer path computes (arXiv 2202.13808).  TEST INFRASTRUCTURE ONLY: it is
+ * called from tests, from the smoke check and from the benchmark's CPU
+ * baseline leg, never from the product path, and it shares no code with the
+ * CUDA library.
+ *
+ * What it states, each from the paper:
+ *   - keep count           Sec. 3.3 ("drop the smallest gamma fraction"), Sec. 4.1
+ *                          ("proportion of 1-gamma"), Table 4 (memory falls by gamma)
+ *   - min-k selection      Sec. 3.3 "Min-K Elements", Sec. 4.1 (largest |a| retained)
+ *   - sparse cache a-hat   Sec. 3.2, a-hat = {a_Xr, X_r} ("coordinate format", Sec. 4.1)
+ *   - recovery R(.)        Sec. 3.2 (dropped indices filled with zero)
+ *   - FC weight gradient   Eq. 6,  g = sum_{n in X_r} grad_z_j^n a_k^n ; App. A.3 G' = (A o D) x Z
+ *   - conv weight gradient Eq. 4-5 (retained term), element-wise mask over the input a
+ *
+ * Floating point: products and sums in double, one rounding to float at the end.
+ * Elements are passed as raw bits (uint16 for bf16, uint32 for fp32); the
+ * ordering key of an element is its bits with the sign bit cleared, so
+ * -0 == +0, Inf is above every finite value and NaN patterns are above Inf.
+ *
+ * Pinned by tests/test_oracle_*.py against: the literal rank definition
+ * (oracle_select_rank) vs the sort (oracle_select_sort) vs numpy's stable
+ * sort; closed-form keep counts; closed-form Gaussian quantiles; all-equal and
+ * strictly-monotone tensors; numpy float64 matmul at gamma = 0; torch's
+ * float64 conv weight gradient; 1x1 conv == FC on the transposed view.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define DT_BF16 0
+#define DT_F32 1
+
+/* ---- element decoding ------------------------------------------------- */
+
+static double bf16_bits_to_double(uint16_t b) {
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+static double f32_bits_to_double(uint32_t u) {
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+static double elem_to_double(const void* x, int64_t i, int dtype) {
+    if (dtype == DT_BF16) return bf16_bits_to_double(((const uint16_t*)x)[i]);
+    return f32_bits_to_double(((const uint32_t*)x)[i]);
+}
+
+/* Ordering key of |x|: the raw bits without the sign bit (Sec. 3.3, absolute magnitude). */
+void oracle_keys(const void* x, int64_t n, int dtype, uint32_t* keys) {
+    for (int64_t i = 0; i < n; ++i) {
+        if (dtype == DT_BF16) keys[i] = ((const uint16_t*)x)[i] & 0x7FFFu;
+        else keys[i] = ((const uint32_t*)x)[i] & 0x7FFFFFFFu;
+    }
+}
+
+/* ---- keep count (Sec. 3.3 / Sec. 4.1 / Table 4) ------------------------ */
+
+/* gamma is the DROPPED fraction.  The number dropped is the smallest integer
+ * not below gamma*n (so at least a gamma fraction goes, never more kept than
+ * the 1-gamma budget); the 1e-6 guard absorbs the binary rounding of gamma
+ * (0.9*10 evaluates to 9.000000000000002 in double). */
+int64_t oracle_keep_count(int64_t n, double gamma) {
+    double d = ceil(gamma * (double)n - 1e-6);
+    if (d < 0.0) d = 0.0;
+    if (d > (double)n) d = (double)n;
+    return n - (int64_t)d;
+}
+
+/* ---- selection --------------------------------------------------------- */
+
+/* Literal definition: rank(i) = #{j : key_j > key_i} + #{j < i : key_j == key_i};
+ * element i is retained iff rank(i) < k.  O(n^2), for small n. */
+void oracle_select_rank(const uint32_t* keys, int64_t n, int64_t k, uint8_t* keep) {
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t rank = 0;
+        for (int64_t j = 0; j < n; ++j) {
+            if (keys[j] > keys[i]) ++rank;
+            else if (keys[j] == keys[i] && j < i) ++rank;
+        }
+        keep[i] = (uint8_t)(rank < k);
+    }
+}
+
+typedef struct {
+    uint32_t key;
+    uint32_t pad;
+    int64_t idx;
+} keyed_t;
+
+static int cmp_key_desc_idx_asc(const void* pa, const void* pb) {
+    const keyed_t* a = (const keyed_t*)pa;
+    const keyed_t* b = (const keyed_t*)pb;
+    if (a->key != b->key) return (a->key > b->key) ? -1 : 1;
+    if (a->idx != b->idx) return (a->idx < b->idx) ? -1 : 1;
+    return 0;
+}
+
+/* Same set by sorting on (key descending, flat index ascending) and taking the
+ * first k.  The comparator is a total order, so the library sort needs no
+ * stability guarantee.  Returns 0, or -1 if memory could not be had. */
+int oracle_select_sort(const uint32_t* keys, int64_t n, int64_t k, uint8_t* keep) {
+    keyed_t* v = (keyed_t*)malloc((size_t)(n > 0 ? n : 1) * sizeof(keyed_t));
+    if (!v) return -1;
+    for (int64_t i = 0; i < n; ++i) {
+        v[i].key = keys[i];
+        v[i].pad = 0;
+        v[i].idx = i;
+    }
+    qsort(v, (size_t)n, sizeof(keyed_t), cmp_key_desc_idx_asc);
+    memset(keep, 0, (size_t)n);
+    for (int64_t r = 0; r < k && r < n; ++r) keep[v[r].idx] = 1;
+    free(v);
+    return 0;
+}
+
+/* D(.) with the min-k strategy on a whole tensor: keys, keep count, selection. */
+int oracle_min_k(const void* x, int64_t n, double gamma, int dtype, uint8_t* keep, int64_t* k_out) {
+    uint32_t* keys = (uint32_t*)malloc((size_t)(n > 0 ? n : 1) * sizeof(uint32_t));
+    if (!keys) return -1;
+    oracle_keys(x, n, dtype, keys);
+    int64_t k = oracle_keep_count(n, gamma);
+    int rc = oracle_select_sort(keys, n, k, keep);
+    free(keys);
+    if (k_out) *k_out = k;
+    return rc;
+}
+
+/* ---- encoders for a-hat = {a_Xr, X_r} (Sec. 3.2) ------------------------ */
+
+/* Occupancy bitmask: element i <-> bit (i mod 32) of 32-bit word (i div 32);
+ * the unused high bits of the last word are 0.  words has ceil(n/32) entries. */
+void oracle_encode_bitmask(const uint8_t* keep, int64_t n, uint32_t* words) {
+    int64_t nw = (n + 31) / 32;
+    for (int64_t w = 0; w < nw; ++w) words[w] = 0;
+    for (int64_t i = 0; i < n; ++i)
+        if (keep[i]) words[i / 32] |= (uint32_t)1 << (i % 32);
+}
+
+/* Retained flat indices in ascending order (the coordinate format's X_r). Returns the count. */
+int64_t oracle_encode_index32(const uint8_t* keep, int64_t n, int32_t* idx) {
+    int64_t c = 0;
+    for (int64_t i = 0; i < n; ++i)
+        if (keep[i]) idx[c++] = (int32_t)i;
+    return c;
+}
+
+/* Retained values a_Xr, raw bits untouched, ascending flat index. Returns the count. */
+int64_t oracle_pack_values(const void* x, const uint8_t* keep, int64_t n, int dtype, void* values) {
+    int64_t c = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (!keep[i]) continue;
+        if (dtype == DT_BF16) ((uint16_t*)values)[c] = ((const uint16_t*)x)[i];
+        else ((uint32_t*)values)[c] = ((const uint32_t*)x)[i];
+        ++c;
+    }
+    return c;
+}
+
+/* offsets[c] = number of retained elements with flat index < c*chunk, for
+ * c = 0 .. ceil(n/chunk)-1 (a seek table into the packed values). */
+void oracle_chunk_offsets(const uint8_t* keep, int64_t n, int64_t chunk, uint32_t* offsets) {
+    int64_t seen = 0; /* retained elements with flat index < i */
+    for (int64_t i = 0; i < n; ++i) {
+        if (i % chunk == 0) offsets[i / chunk] = (uint32_t)seen;
+        seen += keep[i];
+    }
+}
+
+/* ---- recovery R(.) (Sec. 3.2): dropped positions become +0 --------------- */
+
+void oracle_recover_from_bitmask(const void* values, const uint32_t* words, int64_t n, int dtype, void* x_out) {
+    int64_t c = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int kept = (int)((words[i / 32] >> (i % 32)) & 1u);
+        if (dtype == DT_BF16) ((uint16_t*)x_out)[i] = kept ? ((const uint16_t*)values)[c] : 0;
+        else ((uint32_t*)x_out)[i] = kept ? ((const uint32_t*)values)[c] : 0;
+        c += kept;
+    }
+}
+
+void oracle_recover_from_index32(const void* values, const int32_t* idx, int64_t k, int64_t n, int dtype,
+                                 void* x_out) {
+    if (dtype == DT_BF16) memset(x_out, 0, (size_t)n * 2);
+    else memset(x_out, 0, (size_t)n * 4);
+    for (int64_t r = 0; r < k; ++r) {
+        if (dtype == DT_BF16) ((uint16_t*)x_out)[idx[r]] = ((const uint16_t*)values)[r];
+        else ((uint32_t*)x_out)[idx[r]] = ((const uint32_t*)values)[r];
+    }
+}
+
+/* ---- FC weight gradient, Eq. 6 ------------------------------------------ */
+
+/* dw[j*Ca + c] = sum over retained (n, c) of dy[n*Cz + j] * a[n*Ca + c].
+ * Only retained entries are visited; each visits every output row j.
+ * The j loop is the only parallel one (independent outputs). */
+void oracle_fc_weight_grad(const void* dy, const void* x, const uint8_t* keep, int64_t M, int64_t Ca, int64_t Cz,
+                           int dtype, double* dw) {
+    for (int64_t i = 0; i < Cz * Ca; ++i) dw[i] = 0.0;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < Cz; ++j) {
+        for (int64_t n = 0; n < M; ++n) {
+            double g = elem_to_double(dy, n * Cz + j, dtype);
+            for (int64_t c = 0; c < Ca; ++c) {
+                if (!keep[n * Ca + c]) continue;
+                dw[j * Ca + c] += g * elem_to_double(x, n * Ca + c, dtype);
+            }
+        }
+    }
+}
+
+/* One output entry of Eq. 6 at a time, for spot checks at sizes where the full
+ * gradient is too slow: out[s] = dW[js[s], cs[s]]. */
+void oracle_fc_weight_grad_entries(const void* dy, const void* x, const uint8_t* keep, int64_t M, int64_t Ca,
+                                   int64_t Cz, int dtype, const int64_t* js, const int64_t* cs, int64_t ns,
+                                   double* out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < ns; ++s) {
+        int64_t j = js[s], c = cs[s];
+        double acc = 0.0;
+        for (int64_t n = 0; n < M; ++n)
+            if (keep[n * Ca + c]) acc += elem_to_double(dy, n * Cz + j, dtype) * elem_to_double(x, n * Ca + c, dtype);
+        out[s] = acc;
+    }
+}
+
+/* ---- conv weight gradient, Eq. 4-5 (retained term) ----------------------- */
+
+/* dw[j,c,u,v] = sum_{n,y,x} dy[n,j,y,x] * R(a-hat)[n,c, y*stride+u-pad, x*stride+v-pad],
+ * out-of-range input positions contribute 0; NCHW, cross-correlation, groups 1,
+ * dilation 1.  keep is the element-wise mask over the input a. */
+void oracle_conv_weight_grad(const void* dy, const void* x, const uint8_t* keep, int64_t B, int64_t Ca, int64_t H,
+                             int64_t W, int64_t Cz, int64_t R, int64_t S, int64_t stride, int64_t pad, int dtype,
+                             double* dw) {
+    int64_t Ho = (H + 2 * pad - R) / stride + 1;
+    int64_t Wo = (W + 2 * pad - S) / stride + 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < Cz; ++j)
+        for (int64_t c = 0; c < Ca; ++c)
+            for (int64_t u = 0; u < R; ++u)
+                for (int64_t v = 0; v < S; ++v) {
+                    double acc = 0.0;
+                    for (int64_t n = 0; n < B; ++n)
+                        for (int64_t y = 0; y < Ho; ++y)
+                            for (int64_t xx = 0; xx < Wo; ++xx) {
+                                int64_t yi = y * stride + u - pad;
+                                int64_t xi = xx * stride + v - pad;
+                                if (yi < 0 || yi >= H || xi < 0 || xi >= W) continue;
+                                int64_t ia = ((n * Ca + c) * H + yi) * W + xi;
+                                if (!keep[ia]) continue;
+                                int64_t iz = ((n * Cz + j) * Ho + y) * Wo + xx;
+                                acc += elem_to_double(dy, iz, dtype) * elem_to_double(x, ia, dtype);
+                            }
+                    dw[((j * Ca + c) * R + u) * S + v] = acc;
+                }
+}
+
+/* Spot entries of the conv gradient: out[s] = dW[js[s], cs[s], us[s], vs[s]]. */
+void oracle_conv_weight_grad_entries(const void* dy, const void* x, const uint8_t* keep, int64_t B, int64_t Ca,
+                                     int64_t H, int64_t W, int64_t Cz, int64_t R, int64_t S, int64_t stride,
+                                     int64_t pad, int dtype, const int64_t* js, const int64_t* cs, const int64_t* us,
+                                     const int64_t* vs, int64_t ns, double* out) {
+    int64_t Ho = (H + 2 * pad - R) / stride + 1;
+    int64_t Wo = (W + 2 * pad - S) / stride + 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < ns; ++s) {
+        int64_t j = js[s], c = cs[s], u = us[s], v = vs[s];
+        double acc = 0.0;
+        for (int64_t n = 0; n < B; ++n)
+            for (int64_t y = 0; y < Ho; ++y)
+                for (int64_t xx = 0; xx < Wo; ++xx) {
+                    int64_t yi = y * stride + u - pad;
+                    int64_t xi = xx * stride + v - pad;
+                    if (yi < 0 || yi >= H || xi < 0 || xi >= W) continue;
+                    int64_t ia = ((n * Ca + c) * H + yi) * W + xi;
+                    if (!keep[ia]) continue;
+                    int64_t iz = ((n * Cz + j) * Ho + y) * Wo + xx;
+                    acc += elem_to_double(dy, iz, dtype) * elem_to_double(x, ia, dtype);
+                }
+        out[s] = acc;
+    }
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
