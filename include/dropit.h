@@ -1,0 +1,163 @@
+/*
+ * dropit.h - C ABI of the DropIT layer path for NVIDIA B200 (sm_100a).
+ *
+ * DropIT (arXiv 2202.13808) shrinks the activation a that a fully-connected or
+ * convolutional layer caches for its backward pass: the smallest-|a| gamma
+ * fraction of the whole tensor is dropped (Sec. 3.3 "Min-K Elements"), the rest
+ * is kept as a sparse cache a-hat = {a_Xr, X_r} (Sec. 3.2), and the weight
+ * gradient is computed from R(a-hat), the cache with dropped positions read as
+ * zero (Sec. 3.2, Eq. 4-6).
+ *
+ * Conventions for every entry point
+ *  - Pointers marked [device] are CUDA device pointers owned by the caller;
+ *    pointers marked [host] are ordinary host pointers.  The library allocates,
+ *    frees and synchronises nothing: every device call only enqueues work on
+ *    `cuda_stream` (a cudaStream_t passed as void*; NULL = the default stream).
+ *  - Device buffers must be 16-byte aligned.
+ *  - Errors that the host can see (null or misaligned pointers, bad sizes,
+ *    gamma outside [0,1] or NaN, unknown enum, workspace too small) are
+ *    returned before anything is launched.  A CUDA launch error is returned as
+ *    DROPIT_ERR_CUDA.  Device-side waits are bounded; if one runs out the
+ *    kernel stores DROPIT_ERR_TIMEOUT into *dev_status (if given), leaves its
+ *    outputs undefined and returns normally.  dev_status is never cleared by
+ *    the library.
+ *  - gamma is the DROPPED fraction.  n is the number of elements of the layer
+ *    input (every token / pixel / channel of the mini-batch counts: one global
+ *    selection per layer call).  n must be < 2^31.
+ *  - Flat index = row-major offset into the contiguous tensor as passed
+ *    ([M, Ca] for Linear, NCHW for Conv2d).
+ *
+ * Cache layout (what dropit_compress writes, what the gradient calls read)
+ *  - values : the k retained elements, raw bits untouched (-0, NaN payloads and
+ *             denormals survive), in ascending flat index.
+ *  - meta   : DROPIT_FMT_BITMASK - ceil(n/32) little-endian uint32 words, bit
+ *             (i mod 32) of word (i div 32) set iff element i is retained,
+ *             unused high bits of the last word 0;
+ *             DROPIT_FMT_INDEX32 - the k retained flat indices as ascending
+ *             int32 (the coordinate format of Sec. 4.1 / App. A.7).
+ *  - offsets: ceil(n/DROPIT_CHUNK) uint32; offsets[c] = number of retained
+ *             elements with flat index < c*DROPIT_CHUNK (a seek table into
+ *             values; not in the paper, needed to start reading mid-tensor).
+ */
+#ifndef DROPIT_H_
+#define DROPIT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DROPIT_OK = 0,
+    DROPIT_ERR_INVALID_ARG = 1,
+    DROPIT_ERR_UNSUPPORTED = 2,
+    DROPIT_ERR_WORKSPACE = 3,
+    DROPIT_ERR_CUDA = 4,
+    DROPIT_ERR_TIMEOUT = 5
+} dropit_status;
+
+typedef enum { DROPIT_BF16 = 0, DROPIT_F32 = 1 } dropit_dtype;
+typedef enum { DROPIT_FMT_BITMASK = 0, DROPIT_FMT_INDEX32 = 1 } dropit_format;
+
+/* Elements covered by one entry of the offsets table. */
+#define DROPIT_CHUNK 128
+
+/* Library version (major*10000 + minor*100 + patch). [host] */
+int dropit_version(void);
+
+/* Static, human-readable name of a status code. [host] */
+const char* dropit_status_string(dropit_status s);
+
+/*
+ * Number of retained elements for a tensor of n elements at drop ratio gamma:
+ * k = n - ceil(gamma*n - 1e-6), clamped to [0, n], in IEEE double.
+ * (Sec. 3.3: the smallest gamma fraction is dropped; Sec. 4.1: a proportion
+ * 1-gamma is retained; Table 4: the cache shrinks precisely by gamma.  The
+ * paper does not say how to round; this keeps never more than the 1-gamma
+ * budget.)  Returns -1 for n < 0 or gamma outside [0,1] / NaN.  [host]
+ */
+int64_t dropit_keep_count(int64_t n, double gamma);
+
+/*
+ * Byte sizes of the cache buffers and of the scratch workspace that
+ * dropit_compress needs for (n, gamma, dtype, format).  Any output pointer may
+ * be NULL.  Sizes are exact for values/meta/offsets (0 when k = 0 or n = 0);
+ * callers allocate at least that much, 16-byte aligned.  [host]
+ */
+dropit_status dropit_cache_sizes(int64_t n, double gamma, dropit_dtype dtype, dropit_format format,
+                                 size_t* values_bytes, size_t* meta_bytes, size_t* offsets_bytes,
+                                 size_t* workspace_bytes);
+
+/*
+ * D(a) with the min-k strategy (Sec. 3.3, Sec. 4.1): retain the
+ * k = dropit_keep_count(n, gamma) elements of x with the largest |x|, where
+ * |x| is ordered by the raw bits with the sign bit cleared (-0 = +0 < finite <
+ * Inf < NaN patterns) and ties at the threshold go to the LOWER flat index
+ * (the paper leaves ties open).  Writes values / meta / offsets as laid out
+ * above.
+ *   x [device, n elements of dtype, read only]; values, meta, offsets [device,
+ *   written]; workspace [device, scratch of >= workspace_bytes from
+ *   dropit_cache_sizes, contents destroyed, need not be initialised];
+ *   dev_status [device int32, may be NULL].
+ * n = 0 is a no-op.  For k = 0 the mask and offsets are zero-filled.
+ */
+dropit_status dropit_compress(const void* x, int64_t n, double gamma, dropit_dtype dtype, dropit_format format,
+                              void* values, void* meta, uint32_t* offsets, void* workspace, size_t workspace_bytes,
+                              int32_t* dev_status, void* cuda_stream);
+
+/*
+ * R(a-hat) (Sec. 3.2): inflate the cache back to a dense tensor of n elements
+ * with every dropped position +0 and every retained value bit-identical.
+ *   values, meta, offsets [device, read only] as written by dropit_compress for
+ *   the same (n, dtype, format); k = number of retained elements;
+ *   x_dense_out [device, n elements of dtype, written].
+ */
+dropit_status dropit_decompress(const void* values, const void* meta, const uint32_t* offsets, int64_t n, int64_t k,
+                                dropit_dtype dtype, dropit_format format, void* x_dense_out, void* cuda_stream);
+
+/* Scratch bytes that dropit_weight_grad needs for these shapes. [host] */
+dropit_status dropit_weight_grad_workspace(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format,
+                                           size_t* workspace_bytes);
+
+/*
+ * Fully-connected weight gradient from the sparsified cache (Eq. 6; App. A.3
+ * G' = (A o D) x Z):  dw[j, c] = sum over retained (n, c) of dy[n, j] * a[n, c].
+ *   dy [device, M x Cz row-major, dtype]; values/meta/offsets [device] = cache
+ *   of the layer input a [M x Ca row-major]; k its retained count;
+ *   dw [device, Cz x Ca row-major, float]: overwritten, or added to when
+ *   accumulate != 0; workspace [device scratch, contents destroyed].
+ * bf16 inputs multiply on the tensor cores with fp32 accumulation; fp32 inputs
+ * use fp32 FMA.  The summation order is fixed, so results are reproducible
+ * run to run.
+ */
+dropit_status dropit_weight_grad(const void* dy, const void* values, const void* meta, const uint32_t* offsets,
+                                 int64_t M, int64_t Ca, int64_t Cz, int64_t k, dropit_dtype dtype,
+                                 dropit_format format, float* dw, int accumulate, void* workspace,
+                                 size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/* Scratch bytes that dropit_conv_weight_grad needs for these shapes. [host] */
+dropit_status dropit_conv_weight_grad_workspace(int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad,
+                                                dropit_dtype dtype, dropit_format format, size_t* workspace_bytes);
+
+/*
+ * Conv2d weight gradient from the sparsified cache (Eq. 4-5, retained term,
+ * with an element-wise mask over the input a):
+ *   dw[j, c, u, v] = sum_{n, y, x} dy[n, j, y, x] * R(a-hat)[n, c, y*stride + u - pad, x*stride + v - pad],
+ * input positions outside the image contribute 0.  Cross-correlation, NCHW,
+ * groups = 1, dilation must be 1 (anything else: DROPIT_ERR_UNSUPPORTED).
+ *   dy [device, B x Cz x Ho x Wo, dtype] with Ho = (H + 2 pad - R)/stride + 1,
+ *   Wo likewise; values/meta/offsets [device] = cache of a [B x Ca x H x W];
+ *   dw [device, Cz x Ca x R x S, float], overwritten or accumulated into.
+ */
+dropit_status dropit_conv_weight_grad(const void* dy, const void* values, const void* meta, const uint32_t* offsets,
+                                      int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad,
+                                      int dilation, int64_t k, dropit_dtype dtype, dropit_format format, float* dw,
+                                      int accumulate, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                      void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DROPIT_H_ */

@@ -1,0 +1,218 @@
+"""Torch-facing binding of the C ABI in include/dropit.h.
+
+Argument marshalling only: every step (selection, packing, recovery, weight gradients) runs in
+the CUDA library.  torch supplies device memory and the current stream.
+"""
+from __future__ import annotations
+
+import ctypes
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import torch
+
+from . import _lib
+
+BF16, F32 = 0, 1
+FMT_BITMASK, FMT_INDEX32 = 0, 1
+CHUNK = 128
+
+_DTYPE_CODE = {torch.bfloat16: BF16, torch.float32: F32}
+_FMT_CODE = {"bitmask": FMT_BITMASK, "index32": FMT_INDEX32, FMT_BITMASK: FMT_BITMASK, FMT_INDEX32: FMT_INDEX32}
+
+
+class DropITError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s" % (where, dropit_status_string(code)))
+
+
+def library_path() -> str:
+    return _lib.LIB_PATH
+
+
+def dropit_version() -> int:
+    return int(_lib.load().dropit_version())
+
+
+def dropit_status_string(code: int) -> str:
+    return _lib.load().dropit_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise DropITError(code, where)
+
+
+def dropit_keep_count(n: int, gamma: float) -> int:
+    """k = n - ceil(gamma*n - 1e-6): retained elements at drop ratio gamma (Sec. 3.3, Sec. 4.1)."""
+    return int(_lib.load().dropit_keep_count(int(n), float(gamma)))
+
+
+def dropit_cache_sizes(n: int, gamma: float, dtype: int, fmt: int) -> Tuple[int, int, int, int]:
+    """(values_bytes, meta_bytes, offsets_bytes, workspace_bytes) for dropit_compress."""
+    out = [ctypes.c_size_t(0) for _ in range(4)]
+    _check(_lib.load().dropit_cache_sizes(int(n), float(gamma), int(dtype), int(fmt), *[ctypes.byref(o) for o in out]),
+           "dropit_cache_sizes")
+    return tuple(int(o.value) for o in out)
+
+
+@dataclass
+class DropITCache:
+    """a-hat = {a_Xr, X_r} (Sec. 3.2): packed retained values + occupancy mask or int32 indices."""
+    values: torch.Tensor        # k elements, input dtype
+    meta: torch.Tensor          # int32 words: bitmask (ceil(n/32)) or ascending flat indices (k)
+    offsets: torch.Tensor       # int32: retained count before each 128-element chunk
+    n: int
+    k: int
+    shape: Tuple[int, ...]
+    dtype: torch.dtype
+    fmt: int
+    gamma: float
+
+    @property
+    def nbytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in (self.values, self.meta, self.offsets))
+
+
+_status_words = {}
+
+
+def _status_word(device: torch.device) -> torch.Tensor:
+    key = (device.type, device.index)
+    if key not in _status_words:
+        _status_words[key] = torch.zeros(4, dtype=torch.int32, device=device)
+    return _status_words[key]
+
+
+def check_device_status(device=None) -> None:
+    """Synchronise and raise if a kernel reported a bounded wait running out."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    w = _status_word(device)
+    code = int(w[0].item())
+    if code != 0:
+        w.zero_()
+        raise DropITError(code, "device status")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return ctypes.c_void_p(0 if t is None or t.numel() == 0 else t.data_ptr())
+
+
+def _stream_ptr(device) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def _require_cuda(t: torch.Tensor, name: str):
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor (there is no CPU path)" % name)
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    if t.dtype not in _DTYPE_CODE:
+        raise TypeError("%s: dtype %s is not supported (bf16 or fp32)" % (name, t.dtype))
+
+
+def dropit_compress(x: torch.Tensor, gamma: float, fmt="bitmask", workspace: Optional[torch.Tensor] = None) -> DropITCache:
+    """D(a), min-k (Sec. 3.3): retain the k largest-|x| elements of the whole tensor."""
+    _require_cuda(x, "x")
+    lib = _lib.load()
+    fmt = _FMT_CODE[fmt]
+    dt = _DTYPE_CODE[x.dtype]
+    n = x.numel()
+    vb, mb, ob, wb = dropit_cache_sizes(n, gamma, dt, fmt)
+    k = dropit_keep_count(n, gamma)
+    dev = x.device
+    values = torch.empty(vb // x.element_size(), dtype=x.dtype, device=dev)
+    meta = torch.empty(mb // 4, dtype=torch.int32, device=dev)
+    offsets = torch.empty(ob // 4, dtype=torch.int32, device=dev)
+    if workspace is None or workspace.numel() < wb:
+        workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        code = lib.dropit_compress(_ptr(x), n, float(gamma), dt, fmt, _ptr(values), _ptr(meta), _ptr(offsets),
+                                   _ptr(workspace), workspace.numel(), _ptr(_status_word(dev)), _stream_ptr(dev))
+    _check(code, "dropit_compress")
+    return DropITCache(values, meta, offsets, n, k, tuple(x.shape), x.dtype, fmt, float(gamma))
+
+
+def dropit_decompress(cache: DropITCache) -> torch.Tensor:
+    """R(a-hat) (Sec. 3.2): dense tensor, dropped positions +0."""
+    lib = _lib.load()
+    dev = cache.offsets.device if cache.offsets.numel() else cache.values.device
+    out = torch.empty(cache.shape, dtype=cache.dtype, device=dev)
+    with torch.cuda.device(dev):
+        code = lib.dropit_decompress(_ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), cache.n, cache.k,
+                                     _DTYPE_CODE[cache.dtype], cache.fmt, _ptr(out), _stream_ptr(dev))
+    _check(code, "dropit_decompress")
+    return out
+
+
+def dropit_weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(_lib.load().dropit_weight_grad_workspace(M, Ca, Cz, dtype, fmt, ctypes.byref(out)),
+           "dropit_weight_grad_workspace")
+    return int(out.value)
+
+
+def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch.Tensor] = None,
+                       accumulate: bool = False, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Eq. 6: dW[j, c] = sum over retained (n, c) of dY[n, j] a[n, c]; returns fp32 [Cz, Ca]."""
+    _require_cuda(dy, "dy")
+    if dy.dtype != cache.dtype:
+        raise TypeError("dy dtype %s != cache dtype %s" % (dy.dtype, cache.dtype))
+    Ca = cache.shape[-1]
+    M = cache.n // Ca if Ca else 0
+    Cz = dy.shape[-1]
+    if dy.numel() != M * Cz:
+        raise ValueError("dy has %d elements, expected %d x %d" % (dy.numel(), M, Cz))
+    lib = _lib.load()
+    dev = dy.device
+    dt = _DTYPE_CODE[cache.dtype]
+    if out is None:
+        if accumulate:
+            raise ValueError("accumulate=True needs out")
+        out = torch.empty((Cz, Ca), dtype=torch.float32, device=dev)
+    wb = dropit_weight_grad_workspace(M, Ca, Cz, dt, cache.fmt)
+    if workspace is None or workspace.numel() < wb:
+        workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        code = lib.dropit_weight_grad(_ptr(dy), _ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), M, Ca, Cz,
+                                      cache.k, dt, cache.fmt, _ptr(out), int(bool(accumulate)), _ptr(workspace),
+                                      workspace.numel(), _ptr(_status_word(dev)), _stream_ptr(dev))
+    _check(code, "dropit_weight_grad")
+    return out
+
+
+def dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype: int, fmt: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(_lib.load().dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype, fmt,
+                                                         ctypes.byref(out)), "dropit_conv_weight_grad_workspace")
+    return int(out.value)
+
+
+def dropit_conv_weight_grad(dy: torch.Tensor, cache: DropITCache, kernel_size: Tuple[int, int], stride: int = 1,
+                            pad: int = 0, dilation: int = 1, out: Optional[torch.Tensor] = None,
+                            accumulate: bool = False, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Eq. 4-5 retained term: dW[j,c,u,v] from dY [B,Cz,Ho,Wo] and the cache of a [B,Ca,H,W]; fp32."""
+    _require_cuda(dy, "dy")
+    if dy.dtype != cache.dtype:
+        raise TypeError("dy dtype %s != cache dtype %s" % (dy.dtype, cache.dtype))
+    B, Ca, H, W = cache.shape
+    R, S = kernel_size
+    Cz = dy.shape[1]
+    lib = _lib.load()
+    dev = dy.device
+    dt = _DTYPE_CODE[cache.dtype]
+    if out is None:
+        if accumulate:
+            raise ValueError("accumulate=True needs out")
+        out = torch.empty((Cz, Ca, R, S), dtype=torch.float32, device=dev)
+    wb = dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dt, cache.fmt)
+    if workspace is None or workspace.numel() < wb:
+        workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        code = lib.dropit_conv_weight_grad(_ptr(dy), _ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), B, Ca,
+                                           H, W, Cz, R, S, stride, pad, dilation, cache.k, dt, cache.fmt, _ptr(out),
+                                           int(bool(accumulate)), _ptr(workspace), workspace.numel(),
+                                           _ptr(_status_word(dev)), _stream_ptr(dev))
+    _check(code, "dropit_conv_weight_grad")
+    return out

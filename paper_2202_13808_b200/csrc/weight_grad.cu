@@ -1,0 +1,414 @@
+// Fully-connected weight gradient from the sparsified cache (Eq. 6; App. A.3  G' = (A o D) x Z):
+//   dW[j, c] = sum_n dY[n, j] * R(a-hat)[n, c]        dY [M, Cz], a [M, Ca], dW [Cz, Ca]
+//
+// The reduction runs over the token axis n, which is the strided axis of both row-major
+// operands, so for the tensor cores both operands are "MN-major": A = dY^T tile (128 output rows j),
+// B = R(a-hat) tile (256 output columns c), K = 64 tokens per pipeline stage.
+//
+// bf16: tcgen05.mma (kind::f16, fp32 accumulators in TMEM), operands staged in shared memory by
+// TMA in the 128-byte-swizzled canonical layout; one warp issues TMA, one thread issues MMAs,
+// four warps drain TMEM.  Small output matrices are split along n ("split-K"); each split stores
+// its partial tile and the last split to arrive adds the partials in split order, so the
+// summation order is fixed.
+// fp32 (and shapes the TMA path cannot take): an FFMA kernel with 64x64 tiles.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace dropit {
+
+dropit_status decompress_dispatch(const void* values, const void* meta, const uint32_t* offsets, int64_t n, int64_t k,
+                                  dropit_dtype dtype, dropit_format format, void* out, cudaStream_t stream);
+
+// ---------------------------------------------------------------------------------------------
+// Plan
+// ---------------------------------------------------------------------------------------------
+constexpr int kBM = 128;          // output rows (Cz) per tile
+constexpr int kBN = 256;          // output columns (Ca) per tile
+constexpr int kBK = 64;           // tokens per stage
+constexpr int kStages = 4;
+constexpr int kAStageBytes = kBM * kBK * 2;
+constexpr int kBStageBytes = kBN * kBK * 2;
+constexpr int kTcThreads = 192;
+constexpr uint32_t kWaitLimit = 1u << 22;
+
+struct WgPlan {
+    bool tensor_core;
+    int tiles_m, tiles_n, splits, kb_total, kb_per_split;
+    size_t counters_off, counters_bytes;
+    size_t dense_off, dense_bytes;
+    size_t partial_off, partial_bytes;
+    size_t total_bytes;
+};
+
+static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format) {
+    WgPlan p{};
+    p.tensor_core = (dtype == DROPIT_BF16) && (Ca % 8 == 0) && (Cz % 8 == 0);
+    const size_t es = (dtype == DROPIT_BF16) ? 2 : 4;
+    if (p.tensor_core) {
+        p.tiles_m = (int)((Cz + kBM - 1) / kBM);
+        p.tiles_n = (int)((Ca + kBN - 1) / kBN);
+        p.kb_total = (int)((M + kBK - 1) / kBK);
+        const int tiles = p.tiles_m * p.tiles_n;
+        int splits = sm_count() / tiles;
+        if (splits < 1) splits = 1;
+        if (splits > p.kb_total) splits = p.kb_total;
+        p.kb_per_split = (p.kb_total + splits - 1) / splits;
+        p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;   // every split owns >= 1 block
+    } else {
+        p.tiles_m = (int)((Cz + 63) / 64);
+        p.tiles_n = (int)((Ca + 63) / 64);
+        p.splits = 1;
+    }
+    p.counters_off = 0;
+    p.counters_bytes = align_up((size_t)p.tiles_m * p.tiles_n * 4, 256);
+    p.dense_off = p.counters_off + p.counters_bytes;
+    p.dense_bytes = align_up((size_t)M * Ca * es, 256);
+    p.partial_off = p.dense_off + p.dense_bytes;
+    p.partial_bytes = (p.splits > 1) ? align_up((size_t)p.splits * Cz * Ca * 4, 256) : 0;
+    p.total_bytes = p.partial_off + p.partial_bytes;
+    if (p.total_bytes == 0) p.total_bytes = 256;
+    return p;
+}
+
+// ---------------------------------------------------------------------------------------------
+// TMA descriptors (driver entry point fetched at run time; no link-time dependency on libcuda)
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Row-major bf16 matrix [rows, cols]; box = 64 columns (128 bytes) x 64 rows, 128-byte swizzle.
+static bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kBK};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ---------------------------------------------------------------------------------------------
+// tcgen05 kernel
+// ---------------------------------------------------------------------------------------------
+struct TcSmem {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t accum;
+    uint32_t tmem_base;
+    int abort_flag;
+    int is_last;
+};
+constexpr size_t kTcSmemBytes = 1024 + (size_t)kStages * (kAStageBytes + kBStageBytes) + sizeof(TcSmem);
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, int Ca, int Cz,
+             int tiles_n, int splits, int kb_per_split, int kb_total, float* __restrict__ dw, int accumulate,
+             float* __restrict__ partial, uint32_t* counters, int32_t* dev_status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + kStages * kAStageBytes;
+    TcSmem* ctl = reinterpret_cast<TcSmem*>(sB + kStages * kBStageBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int tile = blockIdx.x;
+    const int split = blockIdx.y;
+    const int j0 = (tile / tiles_n) * kBM;
+    const int c0 = (tile % tiles_n) * kBN;
+    const int kb_begin = split * kb_per_split;
+    const int kb_end = min(kb_total, kb_begin + kb_per_split);
+    const int nkb = kb_end - kb_begin;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(&ctl->full[s], 1);
+            ptx::mbar_init(&ctl->empty[s], 1);
+        }
+        ptx::mbar_init(&ctl->accum, 1);
+        ctl->abort_flag = 0;
+        ctl->is_last = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&map_dy);
+        ptx::prefetch_tensormap(&map_x);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&ctl->tmem_base, kBN);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    volatile int* abort_flag = &ctl->abort_flag;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int issued = 0;
+            for (int i = 0; i < nkb && !*abort_flag; ++i) {
+                const int s = i % kStages;
+                if (i >= kStages && !ptx::mbar_wait(&ctl->empty[s], ((i / kStages) - 1) & 1, kWaitLimit)) {
+                    *abort_flag = 1;
+                    break;
+                }
+                ptx::mbar_arrive_expect_tx(&ctl->full[s], kAStageBytes + kBStageBytes);
+                const int k0 = (kb_begin + i) * kBK;
+                uint8_t* a = sA + s * kAStageBytes;
+                uint8_t* b = sB + s * kBStageBytes;
+#pragma unroll
+                for (int g = 0; g < kBM / 64; ++g) ptx::tma_load_2d(a + g * (64 * kBK * 2), &map_dy, j0 + 64 * g, k0, &ctl->full[s]);
+#pragma unroll
+                for (int g = 0; g < kBN / 64; ++g) ptx::tma_load_2d(b + g * (64 * kBK * 2), &map_x, c0 + 64 * g, k0, &ctl->full[s]);
+                issued = i + 1;
+            }
+            if (*abort_flag) {   // let the copies already in flight land before the CTA exits
+                for (int i = max(0, issued - kStages); i < issued; ++i)
+                    ptx::mbar_wait(&ctl->full[i % kStages], (i / kStages) & 1, kWaitLimit);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::make_idesc_bf16(kBM, kBN, true, true);
+            constexpr uint32_t kGroupBytes = 64 * kBK * 2;   // one 64-wide M/N group: kBK rows of 128 bytes
+            bool ok = true;
+            for (int i = 0; i < nkb; ++i) {
+                const int s = i % kStages;
+                if (*abort_flag || !ptx::mbar_wait(&ctl->full[s], (i / kStages) & 1, kWaitLimit)) {
+                    *abort_flag = 1;
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after();
+                const uint32_t a_addr = ptx::smem_u32(sA + s * kAStageBytes);
+                const uint32_t b_addr = ptx::smem_u32(sB + s * kBStageBytes);
+#pragma unroll
+                for (int kk = 0; kk < kBK / 16; ++kk) {
+                    const uint64_t ad = ptx::make_smem_desc_sw128(a_addr + kk * 2048, kGroupBytes, 1024);
+                    const uint64_t bd = ptx::make_smem_desc_sw128(b_addr + kk * 2048, kGroupBytes, 1024);
+                    ptx::umma_bf16(tmem_base, ad, bd, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                }
+                ptx::umma_commit(&ctl->empty[s]);
+            }
+            if (ok) ptx::umma_commit(&ctl->accum);
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> global ----------------
+        const int g = warp & 3;   // TMEM lane quarter this warp may read
+        bool ok = ptx::mbar_wait(&ctl->accum, 0, kWaitLimit);
+        ok = __all_sync(kFullMask, ok) && !*abort_flag;
+        if (!ok) {
+            *abort_flag = 1;
+        } else {
+            ptx::tc_fence_after();
+            const int row = j0 + 32 * g + lane;
+            float* out = (splits > 1) ? (partial + (size_t)split * Cz * Ca) : dw;
+            const bool add = (splits == 1) && accumulate;
+#pragma unroll 1
+            for (int ch = 0; ch < kBN / 32; ++ch) {
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
+                ptx::tmem_ld_wait();
+                if (row < Cz) {
+                    float* dst = out + (size_t)row * Ca + c0 + ch * 32;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        if (c0 + ch * 32 + e + 4 <= Ca) {
+                            float4 v = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
+                                                   __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                            if (add) {
+                                const float4 o = *reinterpret_cast<const float4*>(dst + e);
+                                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                            }
+                            *reinterpret_cast<float4*>(dst + e) = v;
+                        }
+                    }
+                }
+            }
+            if (splits > 1) __threadfence();
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, kBN);
+    }
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
+        return;
+    }
+    if (splits == 1) return;
+
+    // ---- split reduction: the last split to arrive adds the partial tiles in split order ----
+    if (threadIdx.x == 0) {
+        __threadfence();
+        ctl->is_last = (atomicAdd(&counters[tile], 1u) == (uint32_t)splits - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!ctl->is_last) return;
+    __threadfence();
+    const size_t plane = (size_t)Cz * Ca;
+    for (int idx = threadIdx.x; idx < kBM * (kBN / 4); idx += blockDim.x) {
+        const int row = j0 + idx / (kBN / 4);
+        const int col = c0 + (idx % (kBN / 4)) * 4;
+        if (row >= Cz || col + 4 > Ca) continue;
+        const size_t o = (size_t)row * Ca + col;
+        float4 acc = accumulate ? *reinterpret_cast<const float4*>(dw + o) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < splits; ++s) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(partial + s * plane + o));
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        *reinterpret_cast<float4*>(dw + o) = acc;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// FFMA kernel: fp32 inputs, or bf16 shapes that the TMA path cannot take.  64x64 output tile,
+// 16 tokens per step, 4x4 outputs per thread.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+__device__ __forceinline__ float to_float(float f) { return f; }
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+wg_ffma_kernel(const T* __restrict__ dy, const T* __restrict__ xd, int M, int Ca, int Cz, float* __restrict__ dw,
+               int accumulate) {
+    __shared__ float sA[16][64 + 4];
+    __shared__ float sB[16][64 + 4];
+    const int j0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int lr = threadIdx.x >> 4, lc = (threadIdx.x & 15) * 4;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < M; k0 += 16) {
+        const int n = k0 + lr;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = j0 + lc + e, c = c0 + lc + e;
+            sA[lr][lc + e] = (n < M && j < Cz) ? to_float(dy[(size_t)n * Cz + j]) : 0.f;
+            sB[lr][lc + e] = (n < M && c < Ca) ? to_float(xd[(size_t)n * Ca + c]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                a[i] = sA[k][ty * 4 + i];
+                b[i] = sB[k][tx * 4 + i];
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int l = 0; l < 4; ++l) acc[i][l] = fmaf(a[i], b[l], acc[i][l]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int j = j0 + ty * 4 + i, c = c0 + tx * 4 + l;
+            if (j < Cz && c < Ca) {
+                float* d = dw + (size_t)j * Ca + c;
+                *d = accumulate ? (*d + acc[i][l]) : acc[i][l];
+            }
+        }
+}
+
+__global__ void zero_or_keep_kernel(float* dw, int64_t count, int accumulate) {
+    if (accumulate) return;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+        dw[i] = 0.f;
+}
+
+}  // namespace dropit
+
+using namespace dropit;
+
+extern "C" dropit_status dropit_weight_grad_workspace(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype,
+                                                      dropit_format format, size_t* workspace_bytes) {
+    if (M < 0 || Ca <= 0 || Cz <= 0 || M * Ca >= ((int64_t)1 << 31)) return DROPIT_ERR_INVALID_ARG;
+    if ((dtype != DROPIT_BF16 && dtype != DROPIT_F32) || (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32))
+        return DROPIT_ERR_INVALID_ARG;
+    if (workspace_bytes) *workspace_bytes = make_wg_plan(M, Ca, Cz, dtype, format).total_bytes;
+    return DROPIT_OK;
+}
+
+extern "C" dropit_status dropit_weight_grad(const void* dy, const void* values, const void* meta,
+                                            const uint32_t* offsets, int64_t M, int64_t Ca, int64_t Cz, int64_t k,
+                                            dropit_dtype dtype, dropit_format format, float* dw, int accumulate,
+                                            void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                            void* cuda_stream) {
+    if (M < 0 || Ca <= 0 || Cz <= 0 || M * Ca >= ((int64_t)1 << 31) || k < 0 || k > M * Ca) return DROPIT_ERR_INVALID_ARG;
+    if ((dtype != DROPIT_BF16 && dtype != DROPIT_F32) || (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32))
+        return DROPIT_ERR_INVALID_ARG;
+    if (!dw || !is_aligned16(dw)) return DROPIT_ERR_INVALID_ARG;
+    cudaStream_t stream = as_stream(cuda_stream);
+    if (M == 0 || k == 0) {   // empty batch or gamma = 1: the gradient is zero
+        zero_or_keep_kernel<<<sm_count(), 256, 0, stream>>>(dw, Cz * Ca, accumulate);
+        return check_launch();
+    }
+    if (!dy || !values || !meta || !is_aligned16(dy) || !is_aligned16(values) || !is_aligned16(meta))
+        return DROPIT_ERR_INVALID_ARG;
+    if (format == DROPIT_FMT_BITMASK && (!offsets || !is_aligned16(offsets))) return DROPIT_ERR_INVALID_ARG;
+    const WgPlan plan = make_wg_plan(M, Ca, Cz, dtype, format);
+    if (!workspace || !is_aligned16(workspace)) return DROPIT_ERR_INVALID_ARG;
+    if (workspace_bytes < plan.total_bytes) return DROPIT_ERR_WORKSPACE;
+    unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
+    void* dense = ws + plan.dense_off;
+
+    dropit_status s = decompress_dispatch(values, meta, offsets, M * Ca, k, dtype, format, dense, stream);
+    if (s != DROPIT_OK) return s;
+
+    if (!plan.tensor_core) {
+        dim3 grid(plan.tiles_n, plan.tiles_m);
+        if (dtype == DROPIT_BF16)
+            wg_ffma_kernel<uint16_t><<<grid, 256, 0, stream>>>(reinterpret_cast<const uint16_t*>(dy),
+                                                             reinterpret_cast<const uint16_t*>(dense), (int)M, (int)Ca,
+                                                             (int)Cz, dw, accumulate);
+        else
+            wg_ffma_kernel<float><<<grid, 256, 0, stream>>>(reinterpret_cast<const float*>(dy),
+                                                          reinterpret_cast<const float*>(dense), (int)M, (int)Ca,
+                                                          (int)Cz, dw, accumulate);
+        return check_launch();
+    }
+
+    CUtensorMap map_dy, map_x;
+    if (!make_map_2d_bf16(&map_dy, dy, M, Cz) || !make_map_2d_bf16(&map_x, dense, M, Ca)) return DROPIT_ERR_CUDA;
+    uint32_t* counters = reinterpret_cast<uint32_t*>(ws + plan.counters_off);
+    float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
+    if (plan.splits > 1 && cudaMemsetAsync(counters, 0, plan.counters_bytes, stream) != cudaSuccess)
+        return DROPIT_ERR_CUDA;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) !=
+            cudaSuccess)
+            return DROPIT_ERR_CUDA;
+        attr_set = true;
+    }
+    dim3 grid(plan.tiles_m * plan.tiles_n, plan.splits);
+    wg_tc_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n,
+                                                            plan.splits, plan.kb_per_split, plan.kb_total, dw,
+                                                            accumulate, partial, counters, dev_status);
+    return check_launch();
+}

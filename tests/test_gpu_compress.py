@@ -1,0 +1,116 @@
+"""GPU parity: dropit_compress / dropit_decompress against the CPU oracle, bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import dropit_inputs as di
+import oracle
+import paper_2202_13808_b200 as dropit
+from _parity import assert_cache_matches_oracle, np_bits, oracle_cache
+
+pytestmark = pytest.mark.gpu
+
+SMALL = [
+    di.small_linear(1, 1, 1, "bf16", 0.0), di.small_linear(1, 1, 1, "bf16", 0.5), di.small_linear(1, 7, 1, "bf16", 0.5),
+    di.small_linear(3, 11, 1, "bf16", 0.9), di.small_linear(1, 127, 1, "bf16", 0.9), di.small_linear(1, 129, 1, "f32", 0.9),
+    di.small_linear(37, 129, 1, "bf16", 0.9), di.small_linear(64, 768, 1, "bf16", 0.9), di.small_linear(64, 768, 1, "f32", 0.9),
+    di.small_linear(256, 768, 1, "f32", 0.9),                        # the single-Linear fp32 case
+    di.small_linear(1031, 769, 1, "bf16", 0.9),                      # several tiles + ragged tail
+    di.small_linear(1031, 769, 1, "f32", 0.8),
+    di.small_linear(300, 3072, 1, "bf16", 0.9, "gelu"),
+    di.small_linear(512, 768, 1, "bf16", 0.5), di.small_linear(512, 768, 1, "bf16", 0.8),
+    di.small_linear(512, 768, 1, "bf16", 0.0), di.small_linear(512, 768, 1, "bf16", 1.0),
+    di.small_linear(333, 100, 1, "f32", 0.0), di.small_linear(333, 100, 1, "f32", 1.0),
+    di.small_conv(4, 64, 56, 56, 1, 1, 1, gamma=0.8),               # ReLU: half exact zeros
+    di.small_conv(3, 5, 17, 13, 1, 1, 1, gamma=0.3),                 # threshold falls inside the zero ties
+    di.small_conv(3, 5, 17, 13, 1, 1, 1, gamma=0.8, dtype="f32"),
+]
+
+
+@pytest.mark.parametrize("fmt", ["bitmask", "index32"])
+@pytest.mark.parametrize("case", SMALL, ids=lambda c: c.name)
+def test_compress_matches_oracle_small(cuda_device, case, fmt):
+    x = di.make_x(case)
+    bits, dt, keep, k = oracle_cache(x, case.gamma)
+    cache = dropit.dropit_compress(x.to(cuda_device), case.gamma, fmt)
+    dropit.check_device_status(cuda_device)
+    assert_cache_matches_oracle(cache, bits, dt, keep, k, fmt)
+    # R(a-hat): retained values untouched, dropped positions +0
+    rec = dropit.dropit_decompress(cache)
+    expect = np.where(keep == 1, bits, 0).astype(bits.dtype)
+    assert (np_bits(rec) == expect).all()
+
+
+def _special(bits_np, torch_dtype, gamma, fmt, dev):
+    t = torch.from_numpy(bits_np.view(np.int16 if torch_dtype == torch.bfloat16 else np.int32)).view(torch_dtype)
+    dt = oracle.BF16 if torch_dtype == torch.bfloat16 else oracle.F32
+    keep, k = oracle.min_k(bits_np, gamma, dt)
+    cache = dropit.dropit_compress(t.to(dev), gamma, fmt)
+    dropit.check_device_status(dev)
+    assert_cache_matches_oracle(cache, bits_np, dt, keep, k, fmt)
+    return keep
+
+
+@pytest.mark.parametrize("fmt", ["bitmask", "index32"])
+def test_degenerate_tensors(cuda_device, fmt):
+    n = 20011
+    # all equal magnitude, alternating sign: the lowest indices win
+    x = np.full(n, 0x3F80, np.uint16); x[::2] |= 0x8000
+    keep = _special(x, torch.bfloat16, 0.7, fmt, cuda_device)
+    k = int(keep.sum()); assert keep[:k].all()
+    # all zeros (+0 and -0)
+    x = np.zeros(n, np.uint16); x[1::3] = 0x8000
+    _special(x, torch.bfloat16, 0.5, fmt, cuda_device)
+    # strictly increasing magnitude
+    x = (np.arange(1, n + 1, dtype=np.float32) * np.where(np.arange(n) % 2, -1, 1)).astype(np.float32).view(np.uint32)
+    keep = _special(x, torch.float32, 0.9, fmt, cuda_device)
+    assert keep[-int(keep.sum()):].all()
+    # Inf / NaN patterns / denormals / -0 are ordered by raw magnitude bits and stored verbatim
+    rng = np.random.default_rng(3)
+    x = rng.integers(0, 1 << 16, n).astype(np.uint16)
+    _special(x, torch.bfloat16, 0.9, fmt, cuda_device)
+    x = rng.integers(0, 1 << 32, n, dtype=np.uint64).astype(np.uint32)
+    _special(x, torch.float32, 0.6, fmt, cuda_device)
+    # few distinct values: massive ties at the threshold, across many tiles
+    x = rng.integers(0, 3, 100003).astype(np.uint16) * 0x0100 + 0x3F00
+    _special(x, torch.bfloat16, 0.55, fmt, cuda_device)
+    x = (rng.integers(0, 3, 100003).astype(np.uint32) << 23) + 0x3F000000
+    _special(x, torch.float32, 0.55, fmt, cuda_device)
+
+
+def test_empty_tensor_is_a_noop(cuda_device):
+    cache = dropit.dropit_compress(torch.empty(0, dtype=torch.bfloat16, device=cuda_device), 0.5)
+    assert cache.k == 0 and cache.values.numel() == 0 and cache.meta.numel() == 0
+    assert dropit.dropit_decompress(cache).numel() == 0
+
+
+def test_repeat_calls_are_bit_identical(cuda_device):
+    case = di.small_linear(2000, 768, 1, "bf16", 0.9)
+    x = di.make_x(case).to(cuda_device)
+    a = dropit.dropit_compress(x, 0.9)
+    for _ in range(3):
+        b = dropit.dropit_compress(x, 0.9)
+        assert torch.equal(a.values.view(torch.int16), b.values.view(torch.int16))
+        assert torch.equal(a.meta, b.meta) and torch.equal(a.offsets, b.offsets)
+    dropit.check_device_status(cuda_device)
+
+
+FULL = [di.VITB_FC1, di.VITB_FC2, di.R50_CONV1X1, di.R50_CONV3X3,
+        di.with_gamma(di.VITDET_QKV, 0.5), di.with_gamma(di.VITDET_QKV, 0.8), di.VITDET_QKV,
+        di.with_gamma(di.VITDET_FC2, 0.5)]
+
+
+@pytest.mark.parametrize("case", FULL, ids=lambda c: c.name)
+def test_compress_matches_oracle_full_size(cuda_device, case):
+    x = di.make_x(case)
+    bits, dt, keep, k = oracle_cache(x, case.gamma)
+    xg = x.to(cuda_device)
+    cache = dropit.dropit_compress(xg, case.gamma, "bitmask")
+    dropit.check_device_status(cuda_device)
+    assert_cache_matches_oracle(cache, bits, dt, keep, k, "bitmask")
+    rec = dropit.dropit_decompress(cache)
+    assert (np_bits(rec) == np.where(keep == 1, bits, 0).astype(bits.dtype)).all()
+    if case.n <= 40_000_000:
+        cache_i = dropit.dropit_compress(xg, case.gamma, "index32")
+        dropit.check_device_status(cuda_device)
+        assert_cache_matches_oracle(cache_i, bits, dt, keep, k, "index32")

@@ -1,0 +1,87 @@
+"""GPU parity: dropit_weight_grad (Eq. 6) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import dropit_inputs as di
+import oracle
+import paper_2202_13808_b200 as dropit
+from _parity import max_rel_err, oracle_cache
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": 1e-2, "f32": 1e-5}          # max-norm relative error, bf16 inputs / fp32 inputs
+TIGHT = {"bf16": 2e-4, "f32": 1e-5}        # what fp32 accumulation of exact products should reach
+
+SMALL = [
+    di.small_linear(256, 768, 768, "f32", 0.9, dy_std=1.0),           # the single-Linear fp32 configuration
+    di.small_linear(64, 128, 256, "bf16", 0.9),
+    di.small_linear(640, 768, 384, "bf16", 0.9),                       # several k-blocks, 3 column tiles
+    di.small_linear(1000, 512, 384, "bf16", 0.9),                      # ragged token count (1000 = 15*64 + 40)
+    di.small_linear(200, 264, 136, "bf16", 0.5),                       # ragged tiles in both output dims
+    di.small_linear(200, 100, 36, "bf16", 0.5),                        # widths the TMA path cannot take
+    di.small_linear(129, 65, 33, "f32", 0.5, dy_std=1.0),
+    di.small_linear(300, 3072, 128, "bf16", 0.9, "gelu"),
+    di.small_linear(512, 256, 128, "bf16", 0.0),                       # gamma = 0: the dense gradient
+    di.small_linear(512, 256, 128, "bf16", 1.0),                       # gamma = 1: zero gradient
+    di.small_linear(8192, 256, 128, "bf16", 0.9),                      # one tile, deep split along tokens
+]
+
+
+def _run(case, fmt, dev):
+    x, dy = di.make_x(case), di.make_dy(case)
+    bits, dt, keep, k = oracle_cache(x, case.gamma)
+    dyb, _ = oracle.to_bits(dy)
+    cache = dropit.dropit_compress(x.to(dev), case.gamma, fmt)
+    dw = dropit.dropit_weight_grad(dy.to(dev), cache)
+    dropit.check_device_status(dev)
+    return bits, dyb, dt, keep, cache, dw
+
+
+@pytest.mark.parametrize("fmt", ["bitmask", "index32"])
+@pytest.mark.parametrize("case", SMALL, ids=lambda c: c.name)
+def test_weight_grad_matches_oracle(cuda_device, case, fmt):
+    bits, dyb, dt, keep, cache, dw = _run(case, fmt, cuda_device)
+    ref = oracle.fc_weight_grad(dyb, bits, keep, case.M, case.Ca, case.Cz, dt)
+    got = dw.cpu().numpy()
+    assert got.shape == (case.Cz, case.Ca)
+    err = max_rel_err(got, ref)
+    assert err <= TOL[case.dtype], err
+    assert err <= TIGHT[case.dtype], err
+    if case.gamma == 1.0:
+        assert not got.any()
+
+
+def test_accumulate_adds_to_existing_gradient(cuda_device):
+    case = di.small_linear(640, 768, 384, "bf16", 0.9)
+    bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
+    base = torch.full_like(dw, 0.5)
+    out = base.clone()
+    dropit.dropit_weight_grad(di.make_dy(case).to(cuda_device), cache, out=out, accumulate=True)
+    assert torch.allclose(out, dw + base, rtol=1e-6, atol=1e-6)
+    out2 = torch.full_like(dw, 7.0)
+    dropit.dropit_weight_grad(di.make_dy(case).to(cuda_device), cache, out=out2, accumulate=False)
+    assert torch.equal(out2, dw)
+
+
+def test_weight_grad_is_reproducible(cuda_device):
+    case = di.small_linear(8192, 256, 128, "bf16", 0.9)
+    bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
+    dy = di.make_dy(case).to(cuda_device)
+    for _ in range(3):
+        assert torch.equal(dropit.dropit_weight_grad(dy, cache), dw)
+
+
+@pytest.mark.parametrize("case", [di.VITB_FC1, di.VITB_FC2, di.with_gamma(di.VITDET_QKV, 0.8)], ids=lambda c: c.name)
+def test_weight_grad_full_size_sampled_entries(cuda_device, case):
+    bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
+    got = dw.cpu().numpy()
+    rng = np.random.default_rng(0)
+    js = np.concatenate([rng.integers(0, case.Cz, 3000), [0, case.Cz - 1, 0, case.Cz - 1, 127, 128]])
+    cs = np.concatenate([rng.integers(0, case.Ca, 3000), [0, 0, case.Ca - 1, case.Ca - 1, 255, 256]])
+    ref = oracle.fc_weight_grad_entries(dyb, bits, keep, case.M, case.Ca, case.Cz, dt, js, cs)
+    err = np.abs(got[js, cs] - ref).max() / np.abs(ref).max()
+    assert err <= TOL["bf16"] and err <= TIGHT["bf16"], err
+    # a property that holds at any size: column c of dW is zero iff no element of column c was retained
+    col_kept = keep.reshape(case.M, case.Ca).any(axis=0)
+    assert (np.abs(got).max(axis=0)[~col_kept] == 0).all()
