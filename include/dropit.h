@@ -67,6 +67,10 @@ typedef enum { DROPIT_FMT_BITMASK = 0, DROPIT_FMT_INDEX32 = 1 } dropit_format;
 /* Library version (major*10000 + minor*100 + patch). [host] */
 int dropit_version(void);
 
+/* Number of kernels this library has launched in this process since it was loaded (a diagnostic
+ * for benchmarks; memsets are not counted). [host] */
+uint64_t dropit_launch_count(void);
+
 /* Static, human-readable name of a status code. [host] */
 const char* dropit_status_string(dropit_status s);
 

@@ -107,6 +107,7 @@ static int cmp_key_desc_idx_asc(const void* pa, const void* pb) {
  * first k.  The comparator is a total order, so the library sort needs no
  * stability guarantee.  Returns 0, or -1 if memory could not be had. */
 int oracle_select_sort(const uint32_t* keys, int64_t n, int64_t k, uint8_t* keep) {
+    if (n < 0) return -1;
     keyed_t* v = (keyed_t*)malloc((size_t)(n > 0 ? n : 1) * sizeof(keyed_t));
     if (!v) return -1;
     for (int64_t i = 0; i < n; ++i) {

@@ -17,6 +17,7 @@ p_sz = ctypes.POINTER(ctypes.c_size_t)
 # name -> (restype, argtypes); mirrors include/dropit.h
 SIGNATURES = {
     "dropit_version": (c_int, []),
+    "dropit_launch_count": (ctypes.c_uint64, []),
     "dropit_status_string": (ctypes.c_char_p, [c_int]),
     "dropit_keep_count": (c_i64, [c_i64, c_dbl]),
     "dropit_cache_sizes": (c_int, [c_i64, c_dbl, c_int, c_int, p_sz, p_sz, p_sz, p_sz]),

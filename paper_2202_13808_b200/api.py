@@ -35,6 +35,11 @@ def dropit_version() -> int:
     return int(_lib.load().dropit_version())
 
 
+def dropit_launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(_lib.load().dropit_launch_count())
+
+
 def dropit_status_string(code: int) -> str:
     return _lib.load().dropit_status_string(int(code)).decode()
 

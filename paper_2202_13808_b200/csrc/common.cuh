@@ -87,7 +87,12 @@ CompressPlan make_compress_plan(int64_t n, int64_t k, dropit_dtype dtype);
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
+// Kernel launches enqueued by this library since it was loaded (diagnostic counter).
+extern unsigned long long g_launch_count;
+
+// Call once after every kernel launch.
 inline dropit_status check_launch() {
+    ++g_launch_count;
     return cudaGetLastError() == cudaSuccess ? DROPIT_OK : DROPIT_ERR_CUDA;
 }
 

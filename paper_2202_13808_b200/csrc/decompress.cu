@@ -3,6 +3,8 @@
 
 namespace dropit {
 
+unsigned long long g_launch_count = 0;
+
 // One thread per 16-byte output vector.  The number of retained elements before the vector is
 // the chunk's table entry plus the mask bits of the chunk that precede it.
 template <typename Tr>
@@ -108,6 +110,8 @@ extern "C" dropit_status dropit_decompress(const void* values, const void* meta,
 }
 
 extern "C" int dropit_version(void) { return 100; }
+
+extern "C" uint64_t dropit_launch_count(void) { return g_launch_count; }
 
 extern "C" const char* dropit_status_string(dropit_status s) {
     switch (s) {
