@@ -487,6 +487,13 @@ static dropit_status launch_compact(const void* x, const CompressPlan& plan, Sel
 
 }  // namespace dropit
 
+namespace dropit {
+size_t fused_compress_workspace_bytes(int64_t n);
+dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool index32, void* values, void* meta,
+                                  uint32_t* offsets, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                  cudaStream_t stream);
+}  // namespace dropit
+
 using namespace dropit;
 
 extern "C" int64_t dropit_keep_count(int64_t n, double gamma) {
@@ -508,7 +515,8 @@ extern "C" dropit_status dropit_cache_sizes(int64_t n, double gamma, dropit_dtyp
     if (values_bytes) *values_bytes = (size_t)k * es;
     if (meta_bytes) *meta_bytes = (format == DROPIT_FMT_BITMASK) ? (size_t)((n + 31) / 32) * 4 : (size_t)k * 4;
     if (offsets_bytes) *offsets_bytes = (size_t)((n + DROPIT_CHUNK - 1) / DROPIT_CHUNK) * 4;
-    if (workspace_bytes) *workspace_bytes = make_compress_plan(n, k, dtype).total_bytes;
+    if (workspace_bytes)
+        *workspace_bytes = (dtype == DROPIT_BF16) ? fused_compress_workspace_bytes(n) : make_compress_plan(n, k, dtype).total_bytes;
     return DROPIT_OK;
 }
 
@@ -534,8 +542,11 @@ extern "C" dropit_status dropit_compress(const void* x, int64_t n, double gamma,
         if (cudaMemsetAsync(offsets, 0, off_bytes, stream) != cudaSuccess) return DROPIT_ERR_CUDA;
         return DROPIT_OK;
     }
-    const CompressPlan plan = make_compress_plan(n, k, dtype);
     if (!workspace || !is_aligned16(workspace)) return DROPIT_ERR_INVALID_ARG;
+    if (dtype == DROPIT_BF16)
+        return fused_compress_bf16(x, n, k, format == DROPIT_FMT_INDEX32, values, meta, offsets, workspace,
+                                   workspace_bytes, dev_status, stream);
+    const CompressPlan plan = make_compress_plan(n, k, dtype);
     if (workspace_bytes < plan.total_bytes) return DROPIT_ERR_WORKSPACE;
 
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
@@ -544,15 +555,7 @@ extern "C" dropit_status dropit_compress(const void* x, int64_t n, double gamma,
     unsigned long long* desc = reinterpret_cast<unsigned long long*>(ws + plan.desc_offset);
     if (cudaMemsetAsync(ws, 0, plan.total_bytes, stream) != cudaSuccess) return DROPIT_ERR_CUDA;
 
-    dropit_status s;
-    if (dtype == DROPIT_BF16) {
-        s = launch_hist<Bf16Traits, 15, 0, 0, true, true>(x, n, k, st, hist, stream);
-        if (s != DROPIT_OK) return s;
-        if (format == DROPIT_FMT_BITMASK)
-            return launch_compact<Bf16Traits, false>(x, plan, st, desc, values, meta, offsets, dev_status, stream);
-        return launch_compact<Bf16Traits, true>(x, plan, st, desc, values, meta, offsets, dev_status, stream);
-    }
-    s = launch_hist<F32Traits, 11, 20, 0, true, false>(x, n, k, st, hist, stream);
+    dropit_status s = launch_hist<F32Traits, 11, 20, 0, true, false>(x, n, k, st, hist, stream);
     if (s != DROPIT_OK) return s;
     s = launch_hist<F32Traits, 10, 10, 1, false, false>(x, n, k, st, hist + 2048, stream);
     if (s != DROPIT_OK) return s;
