@@ -111,6 +111,37 @@ dropit_status dropit_compress(const void* x, int64_t n, double gamma, dropit_dty
                               void* values, void* meta, uint32_t* offsets, void* workspace, size_t workspace_bytes,
                               int32_t* dev_status, void* cuda_stream);
 
+/* Largest tensor (elements) that dropit_compress_static accepts. */
+#define DROPIT_STATIC_MAX_ELEMS (1 << 28)
+
+/*
+ * dropit_compress for bf16 tensors WITHOUT a workspace argument (the paper has no
+ * counterpart; this exists for callers that must not allocate device memory).
+ * Some callers cannot obtain scratch memory at the moment they need to compress:
+ * a runtime whose device-memory plan is frozen before execution starts, a
+ * plug-in that lives inside a host application and may not touch that
+ * application's allocator (or take its lock from a callback), or an embedded
+ * host that has no allocator to call at all.  For them the scratch that
+ * dropit_compress takes from its `workspace` argument lives in a fixed array
+ * inside the library's device image: dropit_compress_static_scratch_bytes()
+ * bytes (about 400 KB) that every GPU which loads the library holds until the
+ * process exits.
+ *  - Same inputs, outputs, selection rule and cache layout as dropit_compress
+ *    with dtype = DROPIT_BF16; the caller still provides x, values, meta, offsets.
+ *  - n above DROPIT_STATIC_MAX_ELEMS returns DROPIT_ERR_WORKSPACE and launches
+ *    nothing.
+ *  - The call allocates and frees nothing.  The first call on each device looks
+ *    up the array's device address (with that device current); make that first
+ *    call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the last
+ *    call left there; each call clears the part that must start at zero itself.
+ *    Two calls that overlap on the GPU (different streams, no ordering between
+ *    them) would trample each other's scratch: order them.
+ */
+size_t dropit_compress_static_scratch_bytes(void);
+dropit_status dropit_compress_static(const void* x, int64_t n, double gamma, dropit_format format, void* values,
+                                     void* meta, uint32_t* offsets, int32_t* dev_status, void* cuda_stream);
+
 /*
  * R(a-hat) (Sec. 3.2): inflate the cache back to a dense tensor of n elements
  * with every dropped position +0 and every retained value bit-identical.

@@ -786,3 +786,67 @@ dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool inde
 }
 
 }  // namespace dropit
+
+// ---------------------------------------------------------------------------------------------
+// Compression without a caller-provided workspace.
+// ---------------------------------------------------------------------------------------------
+namespace dropit {
+
+// The kernels' scratch (selection state, two key histograms, per-CTA rows) does not grow with the
+// tensor, so one fixed array in device memory can serve.  Every GPU that loads the library holds
+// these bytes until the process exits.
+constexpr size_t kStaticScratchBytes =
+    kStateBytes + 2 * (size_t)kKeySpace * 4 + (size_t)kMaxGrid * 8 + (size_t)kMaxGrid * kRowWords * 4;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// In host code `g_static_scratch` is only a handle for the symbol, not an address a kernel may use:
+// the device address is looked up once per device, with that device current.
+static unsigned char* static_scratch_address() {
+    static unsigned char* cached[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        cached[dev] = reinterpret_cast<unsigned char*>(p);
+    }
+    return cached[dev];
+}
+
+}  // namespace dropit
+
+extern "C" size_t dropit_compress_static_scratch_bytes(void) { return dropit::kStaticScratchBytes; }
+
+extern "C" dropit_status dropit_compress_static(const void* x, int64_t n, double gamma, dropit_format format,
+                                                void* values, void* meta, uint32_t* offsets, int32_t* dev_status,
+                                                void* cuda_stream) {
+    using namespace dropit;
+    if (n < 0 || !(gamma >= 0.0 && gamma <= 1.0)) return DROPIT_ERR_INVALID_ARG;
+    if (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32) return DROPIT_ERR_INVALID_ARG;
+    if (n > DROPIT_STATIC_MAX_ELEMS) return DROPIT_ERR_WORKSPACE;   // beyond what the built-in scratch is stated for
+    if (n == 0) return DROPIT_OK;
+    const int64_t k = dropit_keep_count(n, gamma);
+    if (!x || !offsets || !is_aligned16(x) || !is_aligned16(offsets)) return DROPIT_ERR_INVALID_ARG;
+    if (format == DROPIT_FMT_BITMASK && (!meta || !is_aligned16(meta))) return DROPIT_ERR_INVALID_ARG;
+    if (k > 0 && (!values || !is_aligned16(values))) return DROPIT_ERR_INVALID_ARG;
+    if (k > 0 && format == DROPIT_FMT_INDEX32 && (!meta || !is_aligned16(meta))) return DROPIT_ERR_INVALID_ARG;
+    cudaStream_t stream = as_stream(cuda_stream);
+    if (k == 0) {   // gamma = 1: nothing retained, no scratch involved
+        if (format == DROPIT_FMT_BITMASK &&
+            cudaMemsetAsync(meta, 0, (size_t)((n + 31) / 32) * 4, stream) != cudaSuccess)
+            return DROPIT_ERR_CUDA;
+        if (cudaMemsetAsync(offsets, 0, (size_t)((n + DROPIT_CHUNK - 1) / DROPIT_CHUNK) * 4, stream) != cudaSuccess)
+            return DROPIT_ERR_CUDA;
+        return DROPIT_OK;
+    }
+    if (fused_compress_workspace_bytes(n) > kStaticScratchBytes) return DROPIT_ERR_WORKSPACE;
+    unsigned char* scratch = static_scratch_address();
+    if (!scratch) return DROPIT_ERR_CUDA;
+    // the sample kernel zeroes the part of the scratch that must start at zero on every call
+    return fused_compress_bf16(x, n, k, format == DROPIT_FMT_INDEX32, values, meta, offsets, scratch,
+                               kStaticScratchBytes, dev_status, stream);
+}
+
