@@ -34,11 +34,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within `limit` polls.
+// Bounded wait: false if the phase did not complete within `limit` polls.  Polls back off so that
+// waiting warps do not crowd the shared-memory pipeline of the warps that work.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit) {
-    for (uint32_t i = 0; i < limit; ++i)
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (i > 4) __nanosleep(i > 64 ? 128 : 32);
+    }
     return false;
+}
+// Whole-warp bounded wait: lane 0 polls, then every lane observes the completed phase itself (one
+// successful poll each) so that each thread has its own acquire of the data behind the barrier.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, uint32_t limit) {
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, limit);
+    ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+    if (ok) ok = mbar_wait(bar, parity, 1024);
+    return ok;
 }
 
 // 2-D tiled TMA load, completion signalled on an mbarrier of this CTA.  x is the innermost

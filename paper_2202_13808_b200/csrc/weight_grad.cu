@@ -5,16 +5,15 @@
 // operands, so for the tensor cores both operands are "MN-major": A = dY^T tile (128 output rows j),
 // B = R(a-hat) tile (256 output columns c), K = 64 tokens per pipeline stage.
 //
-// bf16: tcgen05.mma (kind::f16, fp32 accumulators in TMEM), operands staged in shared memory by
-// TMA in the 128-byte-swizzled canonical layout; one warp issues TMA, one thread issues MMAs,
-// four warps drain TMEM.  Small output matrices are split along n ("split-K"); each split stores
-// its partial tile and the last split to arrive adds the partials in split order, so the
-// summation order is fixed.
+// bf16: tcgen05.mma (kind::f16, fp32 accumulators in TMEM), operands staged in shared memory in the
+// 128-byte-swizzled canonical layout.  The bitmask cache is expanded inside the GEMM
+// (weight_grad_fused.cu).  This file holds the variant for the int32-index format and for channel
+// counts that are not a multiple of 128: the cache is first inflated to a dense scratch tensor and
+// both operands arrive by TMA; one warp issues TMA, one thread issues MMAs, four warps drain TMEM.
+// Small output matrices are split along n ("split-K"); each split stores its partial tile and the
+// last split to arrive adds the partials in split order, so the summation order is fixed.
 // fp32 (and shapes the TMA path cannot take): an FFMA kernel with 64x64 tiles.
-#include <cuda.h>
-
-#include "common.cuh"
-#include "sm100_ptx.cuh"
+#include "weight_grad_common.cuh"
 
 namespace dropit {
 
@@ -24,17 +23,12 @@ dropit_status decompress_dispatch(const void* values, const void* meta, const ui
 // ---------------------------------------------------------------------------------------------
 // Plan
 // ---------------------------------------------------------------------------------------------
-constexpr int kBM = 128;          // output rows (Cz) per tile
-constexpr int kBN = 256;          // output columns (Ca) per tile
-constexpr int kBK = 64;           // tokens per stage
 constexpr int kStages = 4;
-constexpr int kAStageBytes = kBM * kBK * 2;
-constexpr int kBStageBytes = kBN * kBK * 2;
 constexpr int kTcThreads = 192;
-constexpr uint32_t kWaitLimit = 1u << 22;
 
 struct WgPlan {
     bool tensor_core;
+    bool fused;               // expand the bitmask cache inside the GEMM (no dense scratch)
     int tiles_m, tiles_n, splits, kb_total, kb_per_split;
     size_t counters_off, counters_bytes;
     size_t dense_off, dense_bytes;
@@ -42,9 +36,10 @@ struct WgPlan {
     size_t total_bytes;
 };
 
-static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format) {
+static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format) {
     WgPlan p{};
     p.tensor_core = (dtype == DROPIT_BF16) && (Ca % 8 == 0) && (Cz % 8 == 0);
+    p.fused = p.tensor_core && format == DROPIT_FMT_BITMASK && (Ca % DROPIT_CHUNK == 0);
     const size_t es = (dtype == DROPIT_BF16) ? 2 : 4;
     if (p.tensor_core) {
         p.tiles_m = (int)((Cz + kBM - 1) / kBM);
@@ -64,7 +59,7 @@ static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype
     p.counters_off = 0;
     p.counters_bytes = align_up((size_t)p.tiles_m * p.tiles_n * 4, 256);
     p.dense_off = p.counters_off + p.counters_bytes;
-    p.dense_bytes = align_up((size_t)M * Ca * es, 256);
+    p.dense_bytes = p.fused ? 0 : align_up((size_t)M * Ca * es, 256);
     p.partial_off = p.dense_off + p.dense_bytes;
     p.partial_bytes = (p.splits > 1) ? align_up((size_t)p.splits * Cz * Ca * 4, 256) : 0;
     p.total_bytes = p.partial_off + p.partial_bytes;
@@ -91,8 +86,7 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Row-major bf16 matrix [rows, cols]; box = 64 columns (128 bytes) x 64 rows, 128-byte swizzle.
-static bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols) {
+bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -212,38 +206,13 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         }
     } else {
         // ---------------- epilogue: TMEM -> global ----------------
-        const int g = warp & 3;   // TMEM lane quarter this warp may read
-        bool ok = ptx::mbar_wait(&ctl->accum, 0, kWaitLimit);
+        bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
         ok = __all_sync(kFullMask, ok) && !*abort_flag;
         if (!ok) {
             *abort_flag = 1;
         } else {
             ptx::tc_fence_after();
-            const int row = j0 + 32 * g + lane;
-            float* out = (splits > 1) ? (partial + (size_t)split * Cz * Ca) : dw;
-            const bool add = (splits == 1) && accumulate;
-#pragma unroll 1
-            for (int ch = 0; ch < kBN / 32; ++ch) {
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
-                ptx::tmem_ld_wait();
-                if (row < Cz) {
-                    float* dst = out + (size_t)row * Ca + c0 + ch * 32;
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        if (c0 + ch * 32 + e + 4 <= Ca) {
-                            float4 v = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
-                                                   __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                            if (add) {
-                                const float4 o = *reinterpret_cast<const float4*>(dst + e);
-                                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-                            }
-                            *reinterpret_cast<float4*>(dst + e) = v;
-                        }
-                    }
-                }
-            }
-            if (splits > 1) __threadfence();
+            epilogue_store_tile(tmem_base, warp, lane, j0, c0, Ca, Cz, split, splits, dw, accumulate, partial);
         }
     }
 
@@ -259,27 +228,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
     }
     if (splits == 1) return;
 
-    // ---- split reduction: the last split to arrive adds the partial tiles in split order ----
-    if (threadIdx.x == 0) {
-        __threadfence();
-        ctl->is_last = (atomicAdd(&counters[tile], 1u) == (uint32_t)splits - 1) ? 1 : 0;
-    }
-    __syncthreads();
-    if (!ctl->is_last) return;
-    __threadfence();
-    const size_t plane = (size_t)Cz * Ca;
-    for (int idx = threadIdx.x; idx < kBM * (kBN / 4); idx += blockDim.x) {
-        const int row = j0 + idx / (kBN / 4);
-        const int col = c0 + (idx % (kBN / 4)) * 4;
-        if (row >= Cz || col + 4 > Ca) continue;
-        const size_t o = (size_t)row * Ca + col;
-        float4 acc = accumulate ? *reinterpret_cast<const float4*>(dw + o) : make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < splits; ++s) {
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(partial + s * plane + o));
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-        }
-        *reinterpret_cast<float4*>(dw + o) = acc;
-    }
+    split_reduce_tile(tile, j0, c0, Ca, Cz, splits, dw, accumulate, partial, counters, &ctl->is_last);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -377,6 +326,14 @@ extern "C" dropit_status dropit_weight_grad(const void* dy, const void* values, 
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
     void* dense = ws + plan.dense_off;
 
+    if (plan.fused) {
+        uint32_t* counters = reinterpret_cast<uint32_t*>(ws + plan.counters_off);
+        float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
+        if (plan.splits > 1 && cudaMemsetAsync(counters, 0, plan.counters_bytes, stream) != cudaSuccess)
+            return DROPIT_ERR_CUDA;
+        return launch_wg_fused(dy, values, meta, offsets, M, Ca, Cz, k, plan.tiles_m, plan.tiles_n, plan.splits,
+                               plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status, stream);
+    }
     dropit_status s = decompress_dispatch(values, meta, offsets, M * Ca, k, dtype, format, dense, stream);
     if (s != DROPIT_OK) return s;
 
