@@ -172,6 +172,20 @@ dropit_status dropit_weight_grad(const void* dy, const void* values, const void*
                                  dropit_format format, float* dw, int accumulate, void* workspace,
                                  size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
+/*
+ * Same result as dropit_weight_grad (Eq. 6), computed WITHOUT inflating the cache to a dense
+ * scratch tensor: mask, seek table and packed values are prefetched into shared memory and the
+ * R(a-hat) tiles (Sec. 3.2) are built there, right in front of the tensor cores.  Needs
+ * dtype = DROPIT_BF16, format = DROPIT_FMT_BITMASK, Ca a multiple of 128 and Cz a multiple of 8;
+ * anything else returns DROPIT_ERR_UNSUPPORTED.  Same arguments and workspace size as
+ * dropit_weight_grad.  On B200 it is currently the slower of the two variants; dropit_weight_grad
+ * chooses between them.
+ */
+dropit_status dropit_weight_grad_fused(const void* dy, const void* values, const void* meta, const uint32_t* offsets,
+                                       int64_t M, int64_t Ca, int64_t Cz, int64_t k, dropit_dtype dtype,
+                                       dropit_format format, float* dw, int accumulate, void* workspace,
+                                       size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
 /* Scratch bytes that dropit_conv_weight_grad needs for these shapes. [host] */
 dropit_status dropit_conv_weight_grad_workspace(int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad,
                                                 dropit_dtype dtype, dropit_format format, size_t* workspace_bytes);

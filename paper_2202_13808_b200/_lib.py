@@ -28,6 +28,8 @@ SIGNATURES = {
     "dropit_weight_grad_workspace": (c_int, [c_i64, c_i64, c_i64, c_int, c_int, p_sz]),
     "dropit_weight_grad": (c_int, [c_vp, c_vp, c_vp, c_vp, c_i64, c_i64, c_i64, c_i64, c_int, c_int, c_vp, c_int,
                                    c_vp, c_sz, c_vp, c_vp]),
+    "dropit_weight_grad_fused": (c_int, [c_vp, c_vp, c_vp, c_vp, c_i64, c_i64, c_i64, c_i64, c_int, c_int, c_vp, c_int,
+                                         c_vp, c_sz, c_vp, c_vp]),
     "dropit_conv_weight_grad_workspace": (c_int, [c_int] * 9 + [c_int, c_int, p_sz]),
     "dropit_conv_weight_grad": (c_int, [c_vp, c_vp, c_vp, c_vp] + [c_int] * 10 + [c_i64, c_int, c_int, c_vp, c_int,
                                         c_vp, c_sz, c_vp, c_vp]),

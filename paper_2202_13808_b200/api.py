@@ -159,8 +159,11 @@ def dropit_weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int)
 
 
 def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch.Tensor] = None,
-                       accumulate: bool = False, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """Eq. 6: dW[j, c] = sum over retained (n, c) of dY[n, j] a[n, c]; returns fp32 [Cz, Ca]."""
+                       accumulate: bool = False, workspace: Optional[torch.Tensor] = None,
+                       fused: bool = False) -> torch.Tensor:
+    """Eq. 6: dW[j, c] = sum over retained (n, c) of dY[n, j] a[n, c]; returns fp32 [Cz, Ca].
+
+    fused=True calls dropit_weight_grad_fused (cache expanded inside the GEMM, no dense scratch)."""
     _require_cuda(dy, "dy")
     if dy.dtype != cache.dtype:
         raise TypeError("dy dtype %s != cache dtype %s" % (dy.dtype, cache.dtype))
@@ -180,10 +183,11 @@ def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch
     if workspace is None or workspace.numel() < wb:
         workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
     with torch.cuda.device(dev):
-        code = lib.dropit_weight_grad(_ptr(dy), _ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), M, Ca, Cz,
+        fn = lib.dropit_weight_grad_fused if fused else lib.dropit_weight_grad
+        code = fn(_ptr(dy), _ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), M, Ca, Cz,
                                       cache.k, dt, cache.fmt, _ptr(out), int(bool(accumulate)), _ptr(workspace),
                                       workspace.numel(), _ptr(_status_word(dev)), _stream_ptr(dev))
-    _check(code, "dropit_weight_grad")
+    _check(code, "dropit_weight_grad_fused" if fused else "dropit_weight_grad")
     return out
 
 

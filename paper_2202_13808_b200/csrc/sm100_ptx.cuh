@@ -43,14 +43,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
     }
     return false;
 }
-// Whole-warp bounded wait: lane 0 polls, then every lane observes the completed phase itself (one
-// successful poll each) so that each thread has its own acquire of the data behind the barrier.
+// Whole-warp bounded wait: lane 0 polls (an mbarrier poll costs on the order of 100 cycles), the
+// warp-level exchange of the result orders the other lanes' later reads after lane 0's acquire.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, uint32_t limit) {
     bool ok = true;
     if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, limit);
-    ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-    if (ok) ok = mbar_wait(bar, parity, 1024);
-    return ok;
+    __syncwarp();
+    return __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
 }
 
 // 2-D tiled TMA load, completion signalled on an mbarrier of this CTA.  x is the innermost

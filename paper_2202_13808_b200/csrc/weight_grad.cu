@@ -23,6 +23,10 @@ dropit_status decompress_dispatch(const void* values, const void* meta, const ui
 // ---------------------------------------------------------------------------------------------
 // Plan
 // ---------------------------------------------------------------------------------------------
+#ifndef DROPIT_FUSED_MIN_TOKENS
+#define DROPIT_FUSED_MIN_TOKENS (1ll << 40)   // never: the dense-scratch variant is faster on every measured shape so far
+#endif
+constexpr int64_t kFusedMinTokens = DROPIT_FUSED_MIN_TOKENS;   // see make_wg_plan
 constexpr int kStages = 4;
 constexpr int kTcThreads = 192;
 
@@ -36,13 +40,18 @@ struct WgPlan {
     size_t total_bytes;
 };
 
-static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format) {
+static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format,
+                           bool force_fused = false) {
     WgPlan p{};
     p.tensor_core = (dtype == DROPIT_BF16) && (Ca % 8 == 0) && (Cz % 8 == 0);
-    p.fused = p.tensor_core && format == DROPIT_FMT_BITMASK && (Ca % DROPIT_CHUNK == 0);
+    // The in-kernel cache expansion (weight_grad_fused.cu) is taken on request (dropit_weight_grad_fused)
+    // or above a token count; on B200 the dense-scratch variant has been faster on every measured shape.
+    const bool fused_ok = p.tensor_core && format == DROPIT_FMT_BITMASK && (Ca % DROPIT_CHUNK == 0);
+    p.fused = fused_ok && (force_fused || M >= kFusedMinTokens);
     const size_t es = (dtype == DROPIT_BF16) ? 2 : 4;
     if (p.tensor_core) {
-        p.tiles_m = (int)((Cz + kBM - 1) / kBM);
+        const int tile_rows = p.fused ? kBM * kFusedAcc : kBM;
+        p.tiles_m = (int)((Cz + tile_rows - 1) / tile_rows);
         p.tiles_n = (int)((Ca + kBN - 1) / kBN);
         p.kb_total = (int)((M + kBK - 1) / kBK);
         const int tiles = p.tiles_m * p.tiles_n;
@@ -299,15 +308,19 @@ extern "C" dropit_status dropit_weight_grad_workspace(int64_t M, int64_t Ca, int
     if (M < 0 || Ca <= 0 || Cz <= 0 || M * Ca >= ((int64_t)1 << 31)) return DROPIT_ERR_INVALID_ARG;
     if ((dtype != DROPIT_BF16 && dtype != DROPIT_F32) || (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32))
         return DROPIT_ERR_INVALID_ARG;
-    if (workspace_bytes) *workspace_bytes = make_wg_plan(M, Ca, Cz, dtype, format).total_bytes;
+    if (workspace_bytes) {   // enough for either variant
+        const size_t a = make_wg_plan(M, Ca, Cz, dtype, format, false).total_bytes;
+        const size_t b = make_wg_plan(M, Ca, Cz, dtype, format, true).total_bytes;
+        *workspace_bytes = a > b ? a : b;
+    }
     return DROPIT_OK;
 }
 
-extern "C" dropit_status dropit_weight_grad(const void* dy, const void* values, const void* meta,
-                                            const uint32_t* offsets, int64_t M, int64_t Ca, int64_t Cz, int64_t k,
-                                            dropit_dtype dtype, dropit_format format, float* dw, int accumulate,
-                                            void* workspace, size_t workspace_bytes, int32_t* dev_status,
-                                            void* cuda_stream) {
+static dropit_status weight_grad_impl(const void* dy, const void* values, const void* meta,
+                                      const uint32_t* offsets, int64_t M, int64_t Ca, int64_t Cz, int64_t k,
+                                      dropit_dtype dtype, dropit_format format, float* dw, int accumulate,
+                                      void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                      void* cuda_stream, bool force_fused) {
     if (M < 0 || Ca <= 0 || Cz <= 0 || M * Ca >= ((int64_t)1 << 31) || k < 0 || k > M * Ca) return DROPIT_ERR_INVALID_ARG;
     if ((dtype != DROPIT_BF16 && dtype != DROPIT_F32) || (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32))
         return DROPIT_ERR_INVALID_ARG;
@@ -320,7 +333,8 @@ extern "C" dropit_status dropit_weight_grad(const void* dy, const void* values, 
     if (!dy || !values || !meta || !is_aligned16(dy) || !is_aligned16(values) || !is_aligned16(meta))
         return DROPIT_ERR_INVALID_ARG;
     if (format == DROPIT_FMT_BITMASK && (!offsets || !is_aligned16(offsets))) return DROPIT_ERR_INVALID_ARG;
-    const WgPlan plan = make_wg_plan(M, Ca, Cz, dtype, format);
+    const WgPlan plan = make_wg_plan(M, Ca, Cz, dtype, format, force_fused);
+    if (force_fused && !plan.fused) return DROPIT_ERR_UNSUPPORTED;
     if (!workspace || !is_aligned16(workspace)) return DROPIT_ERR_INVALID_ARG;
     if (workspace_bytes < plan.total_bytes) return DROPIT_ERR_WORKSPACE;
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
@@ -368,4 +382,22 @@ extern "C" dropit_status dropit_weight_grad(const void* dy, const void* values, 
                                                             plan.splits, plan.kb_per_split, plan.kb_total, dw,
                                                             accumulate, partial, counters, dev_status);
     return check_launch();
+}
+
+extern "C" dropit_status dropit_weight_grad(const void* dy, const void* values, const void* meta,
+                                            const uint32_t* offsets, int64_t M, int64_t Ca, int64_t Cz, int64_t k,
+                                            dropit_dtype dtype, dropit_format format, float* dw, int accumulate,
+                                            void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                            void* cuda_stream) {
+    return weight_grad_impl(dy, values, meta, offsets, M, Ca, Cz, k, dtype, format, dw, accumulate, workspace,
+                            workspace_bytes, dev_status, cuda_stream, false);
+}
+
+extern "C" dropit_status dropit_weight_grad_fused(const void* dy, const void* values, const void* meta,
+                                                  const uint32_t* offsets, int64_t M, int64_t Ca, int64_t Cz,
+                                                  int64_t k, dropit_dtype dtype, dropit_format format, float* dw,
+                                                  int accumulate, void* workspace, size_t workspace_bytes,
+                                                  int32_t* dev_status, void* cuda_stream) {
+    return weight_grad_impl(dy, values, meta, offsets, M, Ca, Cz, k, dtype, format, dw, accumulate, workspace,
+                            workspace_bytes, dev_status, cuda_stream, true);
 }

@@ -8,7 +8,8 @@
 
 namespace dropit {
 
-constexpr int kBM = 128;          // output rows (Cz) per tile
+constexpr int kBM = 128;          // output rows (Cz) per accumulator / MMA
+constexpr int kFusedAcc = 2;      // fused kernel: accumulators per CTA (tile = 256 rows of Cz), fills TMEM
 constexpr int kBN = 256;          // output columns (Ca) per tile
 constexpr int kBK = 64;           // tokens per pipeline stage
 constexpr int kAStageBytes = kBM * kBK * 2;
@@ -51,11 +52,12 @@ __device__ __forceinline__ void epilogue_store_tile(uint32_t tmem_base, int warp
     if (splits > 1) __threadfence();
 }
 
-// Split reduction, called by every thread of the CTA after its partial tile is stored: the last split
-// to arrive adds the partial tiles in split order, so the summation order is fixed.
+// Split reduction, called by every thread of the CTA after its partial tile (tile_rows x 256) is
+// stored: the last split to arrive adds the partial tiles in split order, so the summation order is fixed.
 __device__ __forceinline__ void split_reduce_tile(int tile, int j0, int c0, int Ca, int Cz, int splits,
                                                   float* __restrict__ dw, int accumulate,
-                                                  const float* __restrict__ partial, uint32_t* counters, int* s_is_last) {
+                                                  const float* __restrict__ partial, uint32_t* counters, int* s_is_last,
+                                                  int tile_rows = kBM) {
     if (threadIdx.x == 0) {
         __threadfence();
         *s_is_last = (atomicAdd(&counters[tile], 1u) == (uint32_t)splits - 1) ? 1 : 0;
@@ -64,7 +66,7 @@ __device__ __forceinline__ void split_reduce_tile(int tile, int j0, int c0, int 
     if (!*s_is_last) return;
     __threadfence();
     const size_t plane = (size_t)Cz * Ca;
-    for (int idx = threadIdx.x; idx < kBM * (kBN / 4); idx += blockDim.x) {
+    for (int idx = threadIdx.x; idx < tile_rows * (kBN / 4); idx += blockDim.x) {
         const int row = j0 + idx / (kBN / 4);
         const int col = c0 + (idx % (kBN / 4)) * 4;
         if (row >= Cz || col + 4 > Ca) continue;

@@ -5,15 +5,17 @@
 // so they are prefetched k-blocks ahead into shared-memory rings with per-thread asynchronous copies
 // (cp.async, completion counted on mbarriers):
 //   warp 0  TMA producer: dY tile (A operand) of every stage
-//   warp 1  MMA issuer (one thread), owns the TMEM allocation
+//   warp 1  MMA issuer (one thread), owns the TMEM allocation; every expanded B tile is multiplied
+//           with two dY tiles (256 rows of Cz per CTA, two accumulators = all 512 TMEM columns)
 //   warp 2  meta loader: mask pieces + table entries, up to 6 k-blocks ahead -> meta ring
-//   warps 3, 12  value loaders (half the rows each): once the table entries of a k-block have
+//   warps 3, 20  value loaders (half the rows each): once the table entries of a k-block have
 //           landed, the first 64 packed values of every row (from the 16-byte-aligned start) ->
 //           value ring, eight 16-byte copies per row
-//   warps 4..11  expanders: zero-fill the swizzled B stage and scatter each retained value to its
-//           channel with a 2-byte shared-memory store, then fence to the async proxy and arrive on
-//           the stage's mbarrier.  (A row with more retained values in the tile than the prefetched
-//           window reads the rest from global memory, outside the hot loop.)  Warps 4..7 drain TMEM.
+//   warps 4..19  expanders: a lane owns one 16-byte piece (8 channels) of a row; it gathers its
+//           retained values from the value ring, packs them with zeros and writes the piece of the
+//           swizzled B stage with one 16-byte store, then the warp fences to the async proxy and
+//           arrives on the stage's mbarrier.  (A row with more retained values in the tile than the
+//           prefetched window reads the rest from global memory.)  Warps 4..7 drain TMEM.
 // Waiting warps poll with one lane and back off, so that they do not crowd the shared-memory pipe.
 #include "weight_grad_common.cuh"
 
@@ -22,10 +24,12 @@ namespace dropit {
 namespace {
 
 constexpr int kFStages = 3;                  // A/B pipeline stages
-constexpr int kMetaSlots = 6;                // meta ring depth (k-blocks)
-constexpr int kValSlots = 4;                 // value ring depth (k-blocks)
-constexpr int kExpanders = 8;                // expander warps
-constexpr int kRowsPerExp = kBK / kExpanders;   // 8 rows of a k-block per expander warp
+constexpr int kMetaSlots = 4;                // meta ring depth (k-blocks)
+constexpr int kValSlots = 3;                 // value ring depth (k-blocks)
+constexpr int kExpanders = 16;               // expander warps
+constexpr int kTileRows = kBM * kFusedAcc;   // 256 rows of Cz per CTA: two 128 x 256 accumulators = all 512 TMEM columns
+constexpr int kAFStageBytes = kTileRows * kBK * 2;   // A stage of the fused kernel
+constexpr int kRowsPerExp = kBK / kExpanders;   // 4 rows of a k-block per expander warp
 constexpr int kWinVals = 64;                 // packed values per row held in the value ring
 constexpr int kValLoaders = 2;                // value loader warps: warp 3 and the last warp, half the rows each
 constexpr int kFusedWgThreads = 32 * (4 + kExpanders + (kValLoaders - 1));
@@ -47,8 +51,10 @@ struct FusedCtl {
 constexpr size_t kMaskRingBytes = (size_t)kMetaSlots * kBK * 32;
 constexpr size_t kBaseRingBytes = (size_t)kMetaSlots * kBK * 4;
 constexpr size_t kValRingBytes = (size_t)kValSlots * kBK * kWinVals * 2;
-constexpr size_t kFusedSmemBytes = 1024 + (size_t)kFStages * (kAStageBytes + kBStageBytes) + kMaskRingBytes +
+constexpr size_t kFusedSmemBytes = 1024 + (size_t)kFStages * (kAFStageBytes + kBStageBytes) + kMaskRingBytes +
                                    kBaseRingBytes + kValRingBytes + sizeof(FusedCtl);
+
+static_assert(kFusedSmemBytes <= 232448, "dynamic shared memory of the fused kernel exceeds 227 KB");
 
 // 16-byte copy; with src_bytes = 0 nothing is read and the destination is zero-filled.
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes = 16) {
@@ -81,14 +87,6 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 #define WG_DUMP(cond, slot, ...)
 #endif
 
-template <int N>
-__device__ __forceinline__ bool any_bits(const uint32_t (&b)[N]) {
-    uint32_t o = 0;
-#pragma unroll
-    for (int i = 0; i < N; ++i) o |= b[i];
-    return o != 0;
-}
-
 __global__ void __launch_bounds__(kFusedWgThreads, 1)
 wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __restrict__ values,
                 const uint32_t* __restrict__ mask, const uint32_t* __restrict__ offsets, unsigned long long k_total,
@@ -98,7 +96,7 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
-    uint8_t* sB = sA + kFStages * kAStageBytes;
+    uint8_t* sB = sA + kFStages * kAFStageBytes;
     uint32_t* s_mask = reinterpret_cast<uint32_t*>(sB + kFStages * kBStageBytes);     // [slot][row][8 words]
     uint32_t* s_base = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(s_mask) + kMaskRingBytes);   // [slot][row]
     uint16_t* s_vals = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(s_base) + kBaseRingBytes);   // [slot][row][64]
@@ -108,7 +106,7 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
     const int lane = threadIdx.x & 31;
     const int tile = blockIdx.x;
     const int split = blockIdx.y;
-    const int j0 = (tile / tiles_n) * kBM;
+    const int j0 = (tile / tiles_n) * kTileRows;
     const int c0 = (tile % tiles_n) * kBN;
     const int kb_begin = split * kb_per_split;
     const int kb_end = min(kb_total, kb_begin + kb_per_split);
@@ -135,7 +133,7 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
         ptx::prefetch_tensormap(&map_dy);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(&ctl->tmem_base, kBN);
+        ptx::tmem_alloc(&ctl->tmem_base, kBN * kFusedAcc);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before();
@@ -154,11 +152,11 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
                     *abort_flag = 1;
                     break;
                 }
-                ptx::mbar_arrive_expect_tx(&ctl->full[s], kAStageBytes);
+                ptx::mbar_arrive_expect_tx(&ctl->full[s], kAFStageBytes);
                 const int k0 = (kb_begin + i) * kBK;
-                uint8_t* a = sA + s * kAStageBytes;
+                uint8_t* a = sA + s * kAFStageBytes;
 #pragma unroll
-                for (int g = 0; g < kBM / 64; ++g)
+                for (int g = 0; g < kTileRows / 64; ++g)
                     ptx::tma_load_2d(a + g * (64 * kBK * 2), &map_dy, j0 + 64 * g, k0, &ctl->full[s]);
                 issued = i + 1;
             }
@@ -184,13 +182,17 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
                 }
                 WG_ACC(t_wait_full, c0_);
                 ptx::tc_fence_after();
-                const uint32_t a_addr = ptx::smem_u32(sA + s * kAStageBytes);
+                const uint32_t a_addr = ptx::smem_u32(sA + s * kAFStageBytes);
                 const uint32_t b_addr = ptx::smem_u32(sB + s * kBStageBytes);
 #pragma unroll
                 for (int kk = 0; kk < kBK / 16; ++kk) {
-                    const uint64_t ad = ptx::make_smem_desc_sw128(a_addr + kk * 2048, kGroupBytes, 1024);
                     const uint64_t bd = ptx::make_smem_desc_sw128(b_addr + kk * 2048, kGroupBytes, 1024);
-                    ptx::umma_bf16(tmem_base, ad, bd, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int acc = 0; acc < kFusedAcc; ++acc) {   // the expanded B tile feeds both accumulators
+                        const uint64_t ad =
+                            ptx::make_smem_desc_sw128(a_addr + acc * kAStageBytes + kk * 2048, kGroupBytes, 1024);
+                        ptx::umma_bf16(tmem_base + acc * kBN, ad, bd, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                    }
                 }
                 ptx::umma_commit(&ctl->empty[s]);
             }
@@ -259,44 +261,46 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
     }
     else {
         // ---------------- expanders: mask + packed values -> swizzled B tile ----------------
-        // Lane l owns the 16-byte piece of a row that holds channels c0 + 8l .. c0 + 8l + 7.  The row's
-        // 256 channels are two aligned 128-element chunks of the flat tensor, so the retained count
-        // before lane l is the first chunk's table entry plus the mask bits of the lanes before it.
+        // A warp takes two token rows at a time; lane l owns, in each, the 16-byte piece that holds
+        // channels c0 + 8l .. c0 + 8l + 7 (mask byte l of the row).  The row's 256 channels are two
+        // aligned 128-element chunks of the flat tensor, so the retained count before lane l is the
+        // first chunk's table entry plus the mask bits of the lanes before it (one packed warp scan
+        // for both rows).  Every lane then gathers its up to 8 values from the row's value window
+        // with independent 2-byte shared-memory loads (slot i reads position p + popc(mask below i)),
+        // packs them with zeros and writes the whole piece with one 16-byte store: no zero-fill pass,
+        // no per-element rounds, all lanes busy.
         const int ew = warp - 4;
         const int grp = lane >> 3, piece = lane & 7;
         [[maybe_unused]] long long t_wait_val = 0, t_wait_empty = 0, t_setup = 0, t_rounds = 0, t_tail = 0;
         for (int i = 0; i < nkb; ++i) {
             const int s = i % kFStages, mslot = i % kMetaSlots, vslot = i % kValSlots;
             const long long c0_ = WG_CLK();
-            bool ok = ptx::mbar_wait_warp(&ctl->meta_full[mslot], (i / kMetaSlots) & 1, kWaitLimit) &&
-                      ptx::mbar_wait_warp(&ctl->val_full[vslot], (i / kValSlots) & 1, kWaitLimit);
+            // the value loaders waited for the meta slot before they filled the value slot
+            bool ok = ptx::mbar_wait_warp(&ctl->val_full[vslot], (i / kValSlots) & 1, kWaitLimit);
             WG_ACC(t_wait_val, c0_);
             const long long c1_ = WG_CLK();
             if (ok && i >= kFStages) ok = ptx::mbar_wait_warp(&ctl->empty[s], ((i / kFStages) - 1) & 1, kWaitLimit);
             WG_ACC(t_wait_empty, c1_);
             if (!__all_sync(kFullMask, ok)) *abort_flag = 1;
             if (*abort_flag) break;
-            const long long c2_ = WG_CLK();
+            const long long c3_ = WG_CLK();
+            // 32-bit shared-memory addresses and explicit ld.shared / st.shared keep the address
+            // arithmetic short; all rows of the warp are in flight together
             const uint32_t b_stage = ptx::smem_u32(sB + s * kBStageBytes) + grp * (64 * kBK * 2);
-            const uint32_t* m_row = s_mask + ((size_t)mslot * kBK + ew * kRowsPerExp) * 8;
-            const uint32_t* b_row = s_base + (size_t)mslot * kBK + ew * kRowsPerExp;
-            const uint16_t* v_row = s_vals + ((size_t)vslot * kBK + ew * kRowsPerExp) * kWinVals;
-            // all rows of the warp advance together so that their shared-memory latencies overlap;
-            // two rows share one prefix scan (counts packed in the halves of a word)
-            uint32_t bits[kRowsPerExp], pos[kRowsPerExp], bs[kRowsPerExp], dst[kRowsPerExp], late[kRowsPerExp];
+            const uint32_t m_row = ptx::smem_u32(s_mask + ((size_t)mslot * kBK + ew * kRowsPerExp) * 8) + 4 * (lane >> 2);
+            const uint32_t b_row = ptx::smem_u32(s_base + (size_t)mslot * kBK + ew * kRowsPerExp);
+            const uint32_t v_row = ptx::smem_u32(s_vals + ((size_t)vslot * kBK + ew * kRowsPerExp) * kWinVals);
+            uint32_t m[kRowsPerExp], bs[kRowsPerExp], p0[kRowsPerExp];
 #pragma unroll
             for (int q = 0; q < kRowsPerExp; ++q) {
-                const uint32_t word = m_row[q * 8 + (lane >> 2)];
-                bits[q] = (word >> (8 * (lane & 3))) & 0xFFu;
-                late[q] = 0;
-                bs[q] = b_row[q];
-                const int r = ew * kRowsPerExp + q;
-                dst[q] = b_stage + r * 128 + ((piece ^ (r & 7)) << 4);
-                asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst[q]), "r"(0u));
+                uint32_t word;
+                asm("ld.shared.u32 %0, [%1];" : "=r"(word) : "r"(m_row + q * 32));
+                asm("ld.shared.u32 %0, [%1];" : "=r"(bs[q]) : "r"(b_row + q * 4));
+                m[q] = (word >> (8 * (lane & 3))) & 0xFFu;
             }
 #pragma unroll
-            for (int q = 0; q < kRowsPerExp; q += 2) {
-                const uint32_t cnt2 = __popc(bits[q]) | (__popc(bits[q + 1]) << 16);
+            for (int q = 0; q < kRowsPerExp; q += 2) {   // two rows per prefix scan (counts in the halves of a word)
+                const uint32_t cnt2 = __popc(m[q]) | (__popc(m[q + 1]) << 16);
                 uint32_t inc = cnt2;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -304,48 +308,42 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
                     if (lane >= o) inc += y;
                 }
                 const uint32_t excl2 = inc - cnt2;
-                pos[q] = (bs[q] & 7u) + (excl2 & 0xFFFFu);   // index from the row's 16-byte-aligned start
-                pos[q + 1] = (bs[q + 1] & 7u) + (excl2 >> 16);
+                p0[q] = (bs[q] & 7u) + (excl2 & 0xFFFFu);   // index from the row's 16-byte-aligned start
+                p0[q + 1] = (bs[q + 1] & 7u) + (excl2 >> 16);
             }
-            WG_ACC(t_setup, c2_);
-            const long long c3_ = WG_CLK();
-            while (__any_sync(kFullMask, any_bits<kRowsPerExp>(bits))) {   // one retained element per row and round
-                uint16_t val[kRowsPerExp];
 #pragma unroll
-                for (int q = 0; q < kRowsPerExp; ++q)
-                    val[q] = v_row[q * kWinVals + (pos[q] & (kWinVals - 1))];   // always inside the ring
+            for (int q = 0; q < kRowsPerExp; ++q) {
+                const int r = ew * kRowsPerExp + q;
+                const uint32_t win = v_row + q * (kWinVals * 2);
+                uint32_t v[8];
+                if (p0[q] + __popc(m[q]) <= (uint32_t)kWinVals) {
 #pragma unroll
-                for (int q = 0; q < kRowsPerExp; ++q) {
-                    // branch-free: a lane without a pending element computes a harmless address and
-                    // its store is predicated off
-                    const uint32_t low = bits[q] & (0u - bits[q]);   // lowest pending element (0 if none)
-                    const uint32_t has = low ? 1u : 0u;
-                    const uint32_t in_win = (pos[q] < (uint32_t)kWinVals) ? 1u : 0u;
-                    const uint32_t e2 = (uint32_t)(__ffs(low | 0x100u) - 1) * 2u;
-                    asm volatile(
-                        "{\n\t.reg .pred p;\n\t"
-                        "setp.ne.u32 p, %2, 0;\n\t"
-                        "@p st.shared.u16 [%0], %1;\n\t}"
-                        ::"r"(dst[q] + e2), "h"(val[q]), "r"(has & in_win));
-                    late[q] |= in_win ? 0u : low;   // beyond the prefetched window: fetched after the loop
-                    pos[q] += has;
-                    bits[q] ^= low;
-                }
-            }
-            if (__any_sync(kFullMask, any_bits<kRowsPerExp>(late))) {
-                // rows with more retained values than the prefetched window (rare): the late elements of a
-                // lane are its last ones, at consecutive positions ending at pos - 1
+                    for (int e = 0; e < 8; ++e) {
+                        const uint32_t idx = p0[q] + __popc(m[q] & ((1u << e) - 1u));
+                        uint16_t t;
+                        asm("ld.shared.u16 %0, [%1];" : "=h"(t) : "r"(win + 2 * (idx & (kWinVals - 1))));
+                        v[e] = ((m[q] >> e) & 1u) ? (uint32_t)t : 0u;
+                    }
+                } else {   // a row with more retained values than the prefetched window (rare)
+                    const uint16_t* g = values + (bs[q] & ~7u);
 #pragma unroll
-                for (int q = 0; q < kRowsPerExp; ++q) {
-                    uint32_t p_ = pos[q] - __popc(late[q]);
-                    while (late[q]) {
-                        const int e = __ffs(late[q]) - 1;
-                        const uint16_t v = __ldg(values + (bs[q] & ~7u) + p_);
-                        asm volatile("st.shared.u16 [%0], %1;" ::"r"(dst[q] + 2 * e), "h"(v));
-                        ++p_;
-                        late[q] &= late[q] - 1;
+                    for (int e = 0; e < 8; ++e) {
+                        const uint32_t idx = p0[q] + __popc(m[q] & ((1u << e) - 1u));
+                        v[e] = 0u;
+                        if ((m[q] >> e) & 1u) {
+                            if (idx < (uint32_t)kWinVals) {
+                                uint16_t t;
+                                asm("ld.shared.u16 %0, [%1];" : "=h"(t) : "r"(win + 2 * idx));
+                                v[e] = t;
+                            } else {
+                                v[e] = __ldg(g + idx);
+                            }
+                        }
                     }
                 }
+                const uint32_t dst = b_stage + r * 128 + ((piece ^ (r & 7)) << 4);
+                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[0] | (v[1] << 16)),
+                             "r"(v[2] | (v[3] << 16)), "r"(v[4] | (v[5] << 16)), "r"(v[6] | (v[7] << 16)));
             }
             WG_ACC(t_rounds, c3_);
             const long long c4_ = WG_CLK();
@@ -367,7 +365,10 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
                 *abort_flag = 1;
             } else {
                 ptx::tc_fence_after();
-                epilogue_store_tile(tmem_base, warp, lane, j0, c0, Ca, Cz, split, splits, dw, accumulate, partial);
+#pragma unroll 1
+                for (int acc = 0; acc < kFusedAcc; ++acc)
+                    epilogue_store_tile(tmem_base + acc * kBN, warp, lane, j0 + acc * kBM, c0, Ca, Cz, split, splits, dw,
+                                        accumulate, partial);
             }
         }
     }
@@ -376,14 +377,14 @@ wg_fused_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __re
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, kBN);
+        ptx::tmem_dealloc(tmem_base, kBN * kFusedAcc);
     }
     if (*abort_flag) {
         if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
         return;
     }
     if (splits == 1) return;
-    split_reduce_tile(tile, j0, c0, Ca, Cz, splits, dw, accumulate, partial, counters, &ctl->is_last);
+    split_reduce_tile(tile, j0, c0, Ca, Cz, splits, dw, accumulate, partial, counters, &ctl->is_last, kTileRows);
 }
 
 }  // namespace

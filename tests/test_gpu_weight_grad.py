@@ -52,6 +52,44 @@ def test_weight_grad_matches_oracle(cuda_device, case, fmt):
         assert not got.any()
 
 
+FUSED = [c for c in SMALL if c.dtype == "bf16" and c.Ca % 128 == 0 and c.Cz % 8 == 0] + [
+    di.small_linear(1000, 384, 520, "bf16", 0.9),          # ragged rows of the 256-row tile, 128-channel tail tile
+    di.small_linear(700, 256, 256, "bf16", 0.3),           # dense rows: more retained values than the prefetched window
+    di.small_linear(130, 128, 64, "bf16", 0.0),
+]
+
+
+@pytest.mark.parametrize("case", FUSED, ids=lambda c: c.name)
+def test_fused_weight_grad_matches_oracle(cuda_device, case):
+    """dropit_weight_grad_fused: the cache is expanded inside the GEMM, no dense scratch."""
+    x, dy = di.make_x(case), di.make_dy(case)
+    bits, dt, keep, k = oracle_cache(x, case.gamma)
+    dyb, _ = oracle.to_bits(dy)
+    cache = dropit.dropit_compress(x.to(cuda_device), case.gamma, "bitmask")
+    dw = dropit.dropit_weight_grad(dy.to(cuda_device), cache, fused=True)
+    dropit.check_device_status(cuda_device)
+    ref = oracle.fc_weight_grad(dyb, bits, keep, case.M, case.Ca, case.Cz, dt)
+    err = max_rel_err(dw.cpu().numpy(), ref)
+    assert err <= TOL["bf16"] and err <= TIGHT["bf16"], err
+    # both variants add the same exact bf16 products in fp32; they agree to rounding of the split order
+    dw2 = dropit.dropit_weight_grad(dy.to(cuda_device), cache)
+    assert torch.allclose(dw, dw2, rtol=1e-4, atol=1e-6 * float(dw2.abs().max()))
+    # reproducible run to run
+    assert torch.equal(dw, dropit.dropit_weight_grad(dy.to(cuda_device), cache, fused=True))
+
+
+def test_fused_weight_grad_full_size_and_unsupported(cuda_device):
+    case = di.VITB_FC2
+    bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
+    dwf = dropit.dropit_weight_grad(di.make_dy(case).to(cuda_device), cache, fused=True)
+    dropit.check_device_status(cuda_device)
+    assert torch.allclose(dwf, dw, rtol=1e-4, atol=1e-6 * float(dw.abs().max()))
+    small = di.small_linear(64, 100, 36, "bf16", 0.5)
+    c2 = dropit.dropit_compress(di.make_x(small).to(cuda_device), 0.5, "bitmask")
+    with pytest.raises(dropit.DropITError):
+        dropit.dropit_weight_grad(di.make_dy(small).to(cuda_device), c2, fused=True)
+
+
 def test_accumulate_adds_to_existing_gradient(cuda_device):
     case = di.small_linear(640, 768, 384, "bf16", 0.9)
     bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
