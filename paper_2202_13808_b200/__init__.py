@@ -11,3 +11,4 @@ from .api import (  # noqa: F401
     dropit_decompress, dropit_keep_count, dropit_launch_count, dropit_status_string, dropit_version, dropit_weight_grad,
     dropit_weight_grad_workspace, check_device_status, library_path,
 )
+from .nn import DropITConv2d, DropITConv2dFn, DropITLinear, DropITLinearFn, convert_linear_layers  # noqa: F401
