@@ -4,7 +4,7 @@
 // Every WARP owns one contiguous run of 1024-element blocks and keeps it for the whole kernel, so
 // the ordered compaction needs no block-wide synchronisation and warps drift freely.
 //   sample  (separate 1-CTA kernel) a 16 Ki-element jittered sample brackets the threshold key T
-//           between two keys [lo, hi] (6-sigma margin on the sample rank); it also zeroes the scratch.
+//           between two keys [lo, hi] (6-sigma margin on the sample rank); it also clears the selection state.
 //   phase 1 one read of the tensor: keys above hi are counted in a register, keys inside the band
 //           go to a small per-warp histogram, the rest is ignored (two packed bf16 per 32-bit word
 //           are classified with one add each, so the pass is bound by HBM, not by atomics).
@@ -37,6 +37,9 @@ constexpr int kSampleVecs = 2048;                              // 16384 sampled 
 constexpr int64_t kSampleMinElems = 1 << 19;                   // below this the band is the full key range
 constexpr int kBarrierSpinLimit = 1 << 22;
 constexpr uint32_t kHiBits = 0x80008000u;
+constexpr int kRingDepth = 4;                                  // blocks of a warp's run in flight (cp.async ring)
+constexpr int kRingSlotBytes = kBlkVecs * 16;                  // one block
+constexpr size_t kRingBytes = (size_t)kFusedWarps * kRingDepth * kRingSlotBytes;   // 128 KB
 constexpr int kStageVals = kBlkElems + 16;                     // per-warp staging, values
 constexpr int kStageIdx = kBlkElems + 8;                       // per-warp staging, indices
 
@@ -70,13 +73,15 @@ static FusedPlan make_fused_plan(int64_t n) {
     p.hist_off[0] = kStateBytes;
     p.hist_off[1] = p.hist_off[0] + (size_t)kKeySpace * 4;
     p.agg_off = p.hist_off[1] + (size_t)kKeySpace * 4;
-    p.zero_bytes = p.agg_off + (size_t)kMaxGrid * 8;
-    p.rows_off = p.zero_bytes;                                  // fully written before it is read
+    p.zero_bytes = kStateBytes;                                 // the rest is written before it is read
+    p.rows_off = p.agg_off + (size_t)kMaxGrid * 8;
     p.total_bytes = p.rows_off + (size_t)kMaxGrid * kRowWords * 4;
     return p;
 }
 
 size_t fused_compress_workspace_bytes(int64_t n) { return make_fused_plan(n).total_bytes; }
+
+__device__ __forceinline__ uint32_t ptx_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
     uint32_t v;
@@ -96,6 +101,13 @@ __device__ __forceinline__ void keys_of(const uint4& v, uint32_t (&key)[8]) {
 // Packed compare constant: adding it to two 15-bit keys held in the halves of a 32-bit word sets
 // bit 15 of a half exactly when that key >= bound (no carry crosses the halves).  bound in [0, 32768].
 __device__ __forceinline__ uint32_t ge_const(uint32_t bound) { return ((0x8000u - bound) & 0xFFFFu) * 0x00010001u; }
+
+// Four flags held in bit 15 and bit 31 of two words -> 4 bits in element order (x low, x high, y low, y high):
+// prmt gathers the two high bytes of each word, a multiply lines the four bit-7s up at bits 21..24.
+__device__ __forceinline__ uint32_t flags4(uint32_t x, uint32_t y) {
+    const uint32_t t = (__byte_perm(x, y, 0x7531) >> 7) & 0x01010101u;
+    return ((t * 0x00204081u) >> 21) & 0xFu;
+}
 
 // Exclusive prefix over the block's threads of `v`; also returns the block total.
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s_warp, uint32_t* total) {
@@ -300,6 +312,44 @@ __device__ __forceinline__ void load_block(const uint4* x, int64_t blk, int lane
     }
 }
 
+// The warp's blocks are streamed through a per-warp ring in shared memory fed by cp.async, several
+// blocks ahead, so that enough bytes are in flight per SM without holding them in registers.  Each
+// lane copies and later reads only its own 16-byte vectors, so a cp.async.wait_group is all the
+// synchronisation the ring needs.  `lane_slot` = shared address of the lane's first vector in the slot.
+__device__ __forceinline__ void ring_issue(uint32_t lane_slot, const uint4* x, int64_t blk, int lane, int64_t nvec_full,
+                                           int64_t n) {
+#pragma unroll
+    for (int j = 0; j < kVpl; ++j) {
+        const int64_t vi = blk * kBlkVecs + j * 32 + lane;
+        const uint32_t dst = lane_slot + j * 512;
+        if (vi == nvec_full && (n & 7) != 0) {   // ragged last vector of the tensor: assembled by hand
+            int nv;
+            const uint4 v = load_vec(x, vi, nvec_full, n, &nv);
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                         : "memory");
+        } else {
+            const bool in = vi < nvec_full;   // vectors past the end are zero-filled by the copy itself
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(x + (in ? vi : 0)),
+                         "r"(in ? 16u : 0u)
+                         : "memory");
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void ring_read(uint32_t lane_slot, uint4 (&v)[kVpl]) {
+#pragma unroll
+    for (int j = 0; j < kVpl; ++j)
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w)
+                     : "r"(lane_slot + j * 512)
+                     : "memory");
+}
+// The block issued kRingDepth-1 commits ago has landed.
+__device__ __forceinline__ void ring_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kRingDepth - 1) : "memory"); }
+__device__ __forceinline__ int valid_elems(int64_t vi, int64_t nvec_full, int64_t n) {
+    return vi < nvec_full ? 8 : (vi == nvec_full ? (int)(n & 7) : 0);
+}
+
 // Write the whole 16-byte pieces of a warp's staging buffer and carry the remainder to its front.
 // Slot s of the buffer maps to out[base + s] with base a multiple of PIECE elements; the first
 // `foreign` slots of the very first piece belong to the previous warp and are never written.
@@ -333,14 +383,18 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                       uint32_t* __restrict__ offsets, int32_t* dev_status) {
     extern __shared__ __align__(16) unsigned char fsm[];
     uint32_t* bins = reinterpret_cast<uint32_t*>(fsm);   // general path, phases 1-2: kKeySpace counters
-    uint16_t* s_vals_all = reinterpret_cast<uint16_t*>(fsm);   // phase 3: per-warp staging
-    int32_t* s_idx_all = reinterpret_cast<int32_t*>(fsm + (size_t)kFusedWarps * kStageVals * 2);
-    __shared__ FusedShared sh;
+    // phases 1-2 keep their control block where phase 3 later stages values (phase 3 needs no control block)
+    FusedShared& sh = *reinterpret_cast<FusedShared*>(fsm + kRingBytes);
+    static_assert(sizeof(FusedShared) <= (size_t)kFusedWarps * kStageVals * 2, "control block must fit the staging area");
+    // the input ring shares its memory with the general path's histogram (never live together)
+    uint16_t* s_vals_all = reinterpret_cast<uint16_t*>(fsm + kRingBytes);   // phase 3: per-warp staging
+    int32_t* s_idx_all = reinterpret_cast<int32_t*>(fsm + kRingBytes + (size_t)kFusedWarps * kStageVals * 2);
 
     FusedState* st = reinterpret_cast<FusedState*>(ws);
     unsigned long long* agg = reinterpret_cast<unsigned long long*>(ws + agg_off);
     uint32_t* rows = reinterpret_cast<uint32_t*>(ws + rows_off);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring_lane = ptx_smem(fsm) + (warp * kRingDepth) * kRingSlotBytes + lane * 16;
     const int64_t nvec_full = n / 8;
     const int64_t blocks_total = (n + kBlkElems - 1) / kBlkElems;
     const int64_t blk0 = ((int64_t)blockIdx.x * kFusedWarps + warp) * blocks_per_warp;
@@ -373,25 +427,55 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         uint32_t cnt_hi = 0, cnt_lo = 0;   // keys above the band / keys equal to lo
         auto count_vec = [&](const uint4& v, int nvalid) {
             const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            uint32_t a[4], inb[4], any = 0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint32_t m = w[i] & 0x7FFF7FFFu;
-                const uint32_t a = m + c_hi;                      // bit 15 of a half: key > hi
-                cnt_hi += __popc(a & kHiBits);
-                const uint32_t inb = (m + c_lo) & ~a & kHiBits;   // lo <= key <= hi
-                if (inb) {
-                    if ((inb & 0x8000u) && 2 * i < nvalid) {
-                        const uint32_t d = (m & 0x7FFFu) - lo;
-                        if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
-                    }
-                    if ((inb & 0x80000000u) && 2 * i + 1 < nvalid) {
-                        const uint32_t d = (m >> 16) - lo;
-                        if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
-                    }
+                a[i] = m + c_hi;                       // bit 15 of a half: key > hi
+                inb[i] = (m + c_lo) & ~a[i];           // bit 15 of a half: lo <= key <= hi
+                any |= inb[i];
+            }
+            // keys above the band: one popc per pair of words (the flag bytes gathered by prmt)
+            cnt_hi += __popc(__byte_perm(a[0], a[1], 0x7531) & 0x80808080u) +
+                      __popc(__byte_perm(a[2], a[3], 0x7531) & 0x80808080u);
+            if (any & kHiBits) {   // a few percent of the elements: the band histogram
+                // one pass per in-band element of the lane's vector (a warp needs about two passes), instead
+                // of a divergent test per word and half
+                uint32_t pending = (flags4(inb[0], inb[1]) | (flags4(inb[2], inb[3]) << 4)) & ((1u << nvalid) - 1u);
+                while (pending) {
+                    const uint32_t e = (uint32_t)__ffs(pending) - 1u;
+                    pending &= pending - 1u;
+                    const uint32_t wlo = (e & 2u) ? w[1] : w[0], whi = (e & 2u) ? w[3] : w[2];
+                    const uint32_t ws = (e & 4u) ? whi : wlo;
+                    const uint32_t key = ((e & 1u) ? (ws >> 16) : ws) & 0x7FFFu;
+                    const uint32_t d = key - lo;
+                    if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
                 }
             }
         };
-        {
+        if (narrow) {
+            // stream the run through the ring, kRingDepth-1 blocks ahead
+#pragma unroll
+            for (int d = 0; d < kRingDepth - 1; ++d) {
+                if (blk0 + d < blk1) ring_issue(ring_lane + d * kRingSlotBytes, x, blk0 + d, lane, nvec_full, n);
+                else asm volatile("cp.async.commit_group;" ::: "memory");
+            }
+            int slot = 0, slot_ahead = kRingDepth - 1;
+            for (int64_t blk = blk0; blk < blk1; ++blk) {
+                if (blk + kRingDepth - 1 < blk1)
+                    ring_issue(ring_lane + slot_ahead * kRingSlotBytes, x, blk + kRingDepth - 1, lane, nvec_full, n);
+                else asm volatile("cp.async.commit_group;" ::: "memory");
+                ring_wait();
+                uint4 va[kVpl];
+                ring_read(ring_lane + slot * kRingSlotBytes, va);
+#pragma unroll
+                for (int j = 0; j < kVpl; ++j)
+                    count_vec(va[j], valid_elems(blk * kBlkVecs + j * 32 + lane, nvec_full, n));
+                slot = (slot + 1 == kRingDepth) ? 0 : slot + 1;
+                slot_ahead = (slot_ahead + 1 == kRingDepth) ? 0 : slot_ahead + 1;
+            }
+            asm volatile("cp.async.wait_all;" ::: "memory");
+        } else {
             int64_t blk = blk0;
             for (; blk + kP1Blocks <= blk1; blk += kP1Blocks) {   // 4 loads per lane in flight
                 uint4 va[kP1Blocks][kVpl];
@@ -435,6 +519,14 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                 rows[(size_t)blockIdx.x * kRowWords + threadIdx.x] = v;
             }
         } else {
+            // the global histogram is scratch that nobody cleared: every CTA clears a slice, and one more
+            // grid barrier separates the clearing from the accumulation
+            for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i <= width; i += gridDim.x * blockDim.x) ghist[i] = 0;
+            barrier_target += gridDim.x;
+            if (!grid_barrier(&st->barrier, barrier_target, &sh.ok)) {
+                if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
+                return;
+            }
             for (uint32_t i = threadIdx.x; i <= width; i += blockDim.x) {
                 const uint32_t c = bins[i];
                 if (c) atomicAdd(&ghist[i], c);
@@ -625,38 +717,45 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     uint32_t gpos = run_gt + min(run_eq, q);   // retained elements before this warp's next block
     uint32_t pend = gpos & 7u, foreign = pend;       // staged-but-unwritten values; leading slots not ours
     uint32_t pend_i = gpos & 3u, foreign_i = pend_i;
-    uint4 v[kVpl];
-    int nvalid[kVpl];
-    if (blk0 < blk1) load_block(x, blk0, lane, nvec_full, n, v, nvalid);
+#pragma unroll
+    for (int d = 0; d < kRingDepth - 1; ++d) {
+        if (blk0 + d < blk1) ring_issue(ring_lane + d * kRingSlotBytes, x, blk0 + d, lane, nvec_full, n);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    int slot = 0, slot_ahead = kRingDepth - 1;
     for (int64_t blk = blk0; blk < blk1; ++blk) {
+        if (blk + kRingDepth - 1 < blk1)
+            ring_issue(ring_lane + slot_ahead * kRingSlotBytes, x, blk + kRingDepth - 1, lane, nvec_full, n);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+        ring_wait();
         uint4 cur[kVpl];
+        ring_read(ring_lane + slot * kRingSlotBytes, cur);
+        slot = (slot + 1 == kRingDepth) ? 0 : slot + 1;
+        slot_ahead = (slot_ahead + 1 == kRingDepth) ? 0 : slot_ahead + 1;
+        int nvalid[kVpl];
         uint32_t gt8[kVpl], eq8[kVpl], cnt[kVpl];
 #pragma unroll
         for (int j = 0; j < kVpl; ++j) {
-            cur[j] = v[j];
+            nvalid[j] = valid_elems(blk * kBlkVecs + j * 32 + lane, nvec_full, n);
             const uint32_t w[4] = {cur[j].x, cur[j].y, cur[j].z, cur[j].w};
-            uint32_t g8 = 0, e8 = 0, eany = 0;
-            uint32_t eb[4];
+            uint32_t a[4], eb[4], eany = 0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint32_t m = w[i] & 0x7FFF7FFFu;
-                const uint32_t a = m + c_gt;
-                const uint32_t gb = a & kHiBits;
-                eb[i] = (m + c_ge) & ~a & kHiBits;
+                a[i] = m + c_gt;                        // bit 15 of a half: key > T
+                eb[i] = (m + c_ge) & ~a[i];             // bit 15 of a half: key == T
                 eany |= eb[i];
-                g8 |= ((gb >> (15 - 2 * i)) & (1u << (2 * i))) | ((gb >> (30 - 2 * i)) & (2u << (2 * i)));
             }
-            if (eany) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    e8 |= ((eb[i] >> (15 - 2 * i)) & (1u << (2 * i))) | ((eb[i] >> (30 - 2 * i)) & (2u << (2 * i)));
+            const uint32_t g8 = flags4(a[0], a[1]) | (flags4(a[2], a[3]) << 4);
+            uint32_t e8 = 0;
+            if (eany & kHiBits) {
+                e8 = flags4(eb[0], eb[1]) | (flags4(eb[2], eb[3]) << 4);
                 e8 &= (1u << nvalid[j]) - 1u;   // zero padding past the end must not tie with T = 0
             }
             gt8[j] = g8;
             eq8[j] = e8;
             cnt[j] = __popc(g8) | (__popc(e8) << 16);
         }
-        if (blk + 1 < blk1) load_block(x, blk + 1, lane, nvec_full, n, v, nvalid);   // prefetch
 
         // packed (gt | eq << 16) prefix inside the warp in (j, lane) order
         uint32_t excl[kVpl];
@@ -752,13 +851,14 @@ dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool inde
     const FusedPlan plan = make_fused_plan(n);
     if (workspace_bytes < plan.total_bytes) return DROPIT_ERR_WORKSPACE;
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
-    const size_t smem_hist = (size_t)kKeySpace * 4;
-    size_t smem_idx = (size_t)kFusedWarps * kStageVals * 2 + (size_t)kFusedWarps * kStageIdx * 4;
-    if (smem_idx < smem_hist) smem_idx = smem_hist;   // the general path's histogram lives in the same memory
+    const size_t smem_hist = (size_t)kKeySpace * 4;   // sample kernel: one full key histogram
+    static_assert(kRingBytes >= (size_t)kKeySpace * 4, "the general path's histogram lives in the ring's memory");
+    const size_t smem_mask = kRingBytes + (size_t)kFusedWarps * kStageVals * 2;
+    const size_t smem_idx = smem_mask + (size_t)kFusedWarps * kStageIdx * 4;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(sample_band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_hist) != cudaSuccess ||
-            cudaFuncSetAttribute(fused_compress_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_hist) != cudaSuccess ||
+            cudaFuncSetAttribute(fused_compress_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_mask) != cudaSuccess ||
             cudaFuncSetAttribute(fused_compress_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_idx) != cudaSuccess)
             return DROPIT_ERR_CUDA;
         attr_set = true;
@@ -777,7 +877,7 @@ dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool inde
     int32_t* idxp = index32 ? reinterpret_cast<int32_t*>(meta) : nullptr;
     void* args[] = {&xp, &n, &kk, &bpw, &ws, &h0, &h1, &ao, &ro, &vals, &maskp, &idxp, &offsets, &dev_status};
     const void* fn = index32 ? (const void*)fused_compress_kernel<true> : (const void*)fused_compress_kernel<false>;
-    if (cudaLaunchCooperativeKernel(fn, dim3(plan.grid), dim3(kFusedThreads), args, index32 ? smem_idx : smem_hist,
+    if (cudaLaunchCooperativeKernel(fn, dim3(plan.grid), dim3(kFusedThreads), args, index32 ? smem_idx : smem_mask,
                                     stream) != cudaSuccess) {
         cudaGetLastError();
         return DROPIT_ERR_CUDA;
