@@ -67,8 +67,8 @@ static dropit_status run_decompress(const void* values, const void* meta, const 
     const int64_t cap = (int64_t)sm_count() * 16;
     if (format == DROPIT_FMT_BITMASK) {
         const int64_t nvec = (n + Tr::kVecElems - 1) / Tr::kVecElems;
-        int64_t blocks = (nvec + 255) / 256;
-        if (blocks > cap) blocks = cap;
+        int64_t blocks = (nvec + 255) / 256;   // one vector per thread: short threads, many in flight
+        if (blocks > 0x7FFFFFFF) blocks = 0x7FFFFFFF;
         decompress_bitmask_kernel<Tr><<<(unsigned)blocks, 256, 0, stream>>>(
             reinterpret_cast<const elem_t*>(values), reinterpret_cast<const uint32_t*>(meta), offsets, n,
             reinterpret_cast<elem_t*>(out));

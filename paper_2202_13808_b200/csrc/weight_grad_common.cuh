@@ -66,17 +66,36 @@ __device__ __forceinline__ void split_reduce_tile(int tile, int j0, int c0, int 
     if (!*s_is_last) return;
     __threadfence();
     const size_t plane = (size_t)Cz * Ca;
-    for (int idx = threadIdx.x; idx < tile_rows * (kBN / 4); idx += blockDim.x) {
-        const int row = j0 + idx / (kBN / 4);
-        const int col = c0 + (idx % (kBN / 4)) * 4;
-        if (row >= Cz || col + 4 > Ca) continue;
-        const size_t o = (size_t)row * Ca + col;
-        float4 acc = accumulate ? *reinterpret_cast<const float4*>(dw + o) : make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < splits; ++s) {
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(partial + s * plane + o));
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    // several float4 columns per thread and all splits' loads of them in flight together: the last CTA
+    // of a tile runs this alone, so its memory latency is on the kernel's critical path
+    constexpr int U = 4;
+    const int total = tile_rows * (kBN / 4);
+    for (int base = threadIdx.x; base < total; base += blockDim.x * U) {
+        float4 acc[U];
+        size_t o[U];
+        bool ok[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int idx = base + u * blockDim.x;
+            const int row = j0 + idx / (kBN / 4);
+            const int col = c0 + (idx % (kBN / 4)) * 4;
+            ok[u] = idx < total && row < Cz && col + 4 <= Ca;
+            o[u] = ok[u] ? ((size_t)row * Ca + col) : 0;
+            acc[u] = (accumulate && ok[u]) ? *reinterpret_cast<const float4*>(dw + o[u]) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        *reinterpret_cast<float4*>(dw + o) = acc;
+        for (int s = 0; s < splits; ++s) {   // fixed order over the splits
+            float4 v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                v[u] = ok[u] ? __ldcg(reinterpret_cast<const float4*>(partial + s * plane + o[u])) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (ok[u]) *reinterpret_cast<float4*>(dw + o[u]) = acc[u];
     }
 }
 
