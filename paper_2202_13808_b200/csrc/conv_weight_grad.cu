@@ -10,6 +10,14 @@ namespace dropit {
 dropit_status decompress_dispatch(const void* values, const void* meta, const uint32_t* offsets, int64_t n, int64_t k,
                                   dropit_dtype dtype, dropit_format format, void* out, cudaStream_t stream);
 
+// Tensor-core path (bf16, stride 1, rows a multiple of 8 pixels), defined in conv_weight_grad_tc.cu.
+size_t conv_tc_workspace_bytes(int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad,
+                               dropit_dtype dtype);
+dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, const uint32_t* offsets, int B, int Ca,
+                          int H, int W, int Cz, int R, int S, int stride, int pad, int64_t k, dropit_format format,
+                          float* dw, int accumulate, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                          cudaStream_t stream);
+
 constexpr int kConvTJ = 32;     // output channels per block
 constexpr int kConvTC = 8;      // input channels per block
 constexpr int kConvMaxUV = 9;   // filter taps accumulated per sweep
@@ -148,8 +156,9 @@ extern "C" dropit_status dropit_conv_weight_grad_workspace(int B, int Ca, int H,
     if ((dtype != DROPIT_BF16 && dtype != DROPIT_F32) || (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32))
         return DROPIT_ERR_INVALID_ARG;
     if (workspace_bytes) {
+        const size_t tc = (B > 0) ? conv_tc_workspace_bytes(B, Ca, H, W, Cz, R, S, stride, pad, dtype) : 0;
         const ConvPlan p = make_conv_plan(B, Ca, H, W, Cz, R, S, stride, pad, dtype);
-        *workspace_bytes = p.total_bytes ? p.total_bytes : 256;
+        *workspace_bytes = tc ? tc : (p.total_bytes ? p.total_bytes : 256);
     }
     return DROPIT_OK;
 }
@@ -160,7 +169,6 @@ extern "C" dropit_status dropit_conv_weight_grad(const void* dy, const void* val
                                                  dropit_dtype dtype, dropit_format format, float* dw, int accumulate,
                                                  void* workspace, size_t workspace_bytes, int32_t* dev_status,
                                                  void* cuda_stream) {
-    (void)dev_status;
     dropit_status s = conv_check_shape(B, Ca, H, W, Cz, R, S, stride, pad);
     if (s != DROPIT_OK) return s;
     if ((dtype != DROPIT_BF16 && dtype != DROPIT_F32) || (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32))
@@ -177,9 +185,12 @@ extern "C" dropit_status dropit_conv_weight_grad(const void* dy, const void* val
     if (!dy || !values || !meta || !is_aligned16(dy) || !is_aligned16(values) || !is_aligned16(meta))
         return DROPIT_ERR_INVALID_ARG;
     if (format == DROPIT_FMT_BITMASK && (!offsets || !is_aligned16(offsets))) return DROPIT_ERR_INVALID_ARG;
+    if (!workspace || !is_aligned16(workspace)) return DROPIT_ERR_INVALID_ARG;
+    if (conv_tc_workspace_bytes(B, Ca, H, W, Cz, R, S, stride, pad, dtype) != 0)
+        return conv_tc_run(dy, values, meta, offsets, B, Ca, H, W, Cz, R, S, stride, pad, k, format, dw, accumulate,
+                           workspace, workspace_bytes, dev_status, stream);
     const ConvPlan plan = make_conv_plan(B, Ca, H, W, Cz, R, S, stride, pad, dtype);
     if (plan.smem_bytes > 200 * 1024) return DROPIT_ERR_UNSUPPORTED;
-    if (!workspace || !is_aligned16(workspace)) return DROPIT_ERR_INVALID_ARG;
     if (workspace_bytes < plan.total_bytes) return DROPIT_ERR_WORKSPACE;
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
     void* dense = ws + plan.dense_off;

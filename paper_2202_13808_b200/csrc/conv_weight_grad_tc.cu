@@ -1,0 +1,405 @@
+// Conv2d weight gradient on the tensor cores (Eq. 4-5, retained term), bf16, stride 1:
+//   dW[j,c,u,v] = sum_{n,y,x} dY[n,j,y,x] * R(a-hat)[n,c, y+u-pad, x+v-pad]
+// One implicit GEMM per filter tap (u,v): M = output channels j, N = input channels c, and the
+// reduction runs over (n, y, x) with x innermost, which is the contiguous axis of both NCHW operands,
+// so both are K-major for tcgen05.  A k-block is one image row: 64 x-positions of one (n, y).
+// TMA tiles (4-D maps {W, H, C, B}, 128-byte swizzle) bring 128 rows of dY and BN rows of the input;
+// the tap's vertical offset u-pad is a TMA coordinate (rows outside the image are zero-filled by the
+// hardware), the horizontal offset v-pad cannot be one (a TMA tile must start on a 16-byte boundary),
+// so the dense scratch holds one copy of R(a-hat) per horizontal offset, shifted by whole pixels.
+// Every split of the reduction stores its partial tile; a second kernel adds them in split order.
+#include "weight_grad_common.cuh"
+
+namespace dropit {
+
+dropit_status decompress_dispatch(const void* values, const void* meta, const uint32_t* offsets, int64_t n, int64_t k,
+                                  dropit_dtype dtype, dropit_format format, void* out, cudaStream_t stream);
+
+namespace {
+
+constexpr int kCStages = 4;
+constexpr int kCThreads = 192;
+constexpr int kMaxTapsX = 7;          // widest filter the tensor-core path takes
+
+struct ConvMaps {
+    CUtensorMap dy;
+    CUtensorMap x[kMaxTapsX];        // one per horizontal tap offset
+};
+
+struct ConvTcSmem {
+    uint64_t full[kCStages];
+    uint64_t empty[kCStages];
+    uint64_t accum;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+constexpr size_t kConvTcSmemBytes = 1024 + (size_t)kCStages * (kAStageBytes + kBStageBytes) + sizeof(ConvTcSmem);
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn conv_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// NCHW bf16 tensor [B, C, H, W]; box = xb x-positions x yb rows x `rows` channels x 1 image.  A box may
+// reach outside the tensor in any dimension: those elements arrive as zeros.
+bool make_map_nchw(CUtensorMap* map, const void* base, int B, int C, int H, int W, int xb, int yb, int rows) {
+    EncodeTiledFn fn = conv_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)C, (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)W * 2, (cuuint64_t)H * W * 2, (cuuint64_t)C * H * W * 2};
+    cuuint32_t box[4] = {(cuuint32_t)xb, (cuuint32_t)yb, (cuuint32_t)rows, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(ptx::smem_u32(smem_dst)), "l"(map), "r"(ptx::smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+// One pass over R(a-hat) writes every horizontally shifted copy the filter needs:
+//   out_shift[n,c,y,x] = in[n,c,y,x + shift]  (0 outside the row)  for every shift != 0 with a destination.
+// A thread owns 8 pixels (16 bytes, rows are multiples of 8 pixels) and its two neighbour groups.
+struct ShiftDst {
+    uint4* out[2 * kMaxTapsX - 1];   // indexed by shift + kMaxTapsX - 1; null where the filter has no such tap
+};
+
+__global__ void __launch_bounds__(256)
+shift_copies_kernel(const uint4* __restrict__ in, ShiftDst dst, int64_t groups, int groups_per_row) {
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += (int64_t)gridDim.x * blockDim.x) {
+        const int gx = (int)(g % groups_per_row);
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+        const uint4 cur = __ldg(in + g);
+        const uint4 prev = gx > 0 ? __ldg(in + g - 1) : zero;
+        const uint4 next = gx + 1 < groups_per_row ? __ldg(in + g + 1) : zero;
+        const uint32_t w[12] = {prev.x, prev.y, prev.z, prev.w, cur.x, cur.y, cur.z, cur.w, next.x, next.y, next.z, next.w};
+#pragma unroll
+        for (int sh = -(kMaxTapsX - 1); sh <= kMaxTapsX - 1; ++sh) {
+            uint4* out = dst.out[sh + kMaxTapsX - 1];
+            if (sh == 0 || out == nullptr) continue;
+            const int s = 8 + sh;                 // first window pixel of the shifted group
+            uint4 o;
+            if ((s & 1) == 0) {
+                o = make_uint4(w[s / 2], w[s / 2 + 1], w[s / 2 + 2], w[s / 2 + 3]);
+            } else {
+                const int a = (s - 1) / 2;
+                o = make_uint4(__funnelshift_r(w[a], w[a + 1], 16), __funnelshift_r(w[a + 1], w[a + 2], 16),
+                               __funnelshift_r(w[a + 2], w[a + 3], 16), __funnelshift_r(w[a + 3], w[a + 4], 16));
+            }
+            out[g] = o;
+        }
+    }
+}
+
+// dw[j,c,u,v] (=|+=) sum over splits of partial[split][tap][j][c]
+__global__ void __launch_bounds__(256)
+conv_tc_reduce_kernel(const float* __restrict__ partial, int splits, int Cz, int Ca, int taps, float* __restrict__ dw,
+                      int accumulate) {
+    const int64_t plane = (int64_t)taps * Cz * Ca;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < plane; i += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % Ca);
+        const int j = (int)((i / Ca) % Cz);
+        const int tap = (int)(i / ((int64_t)Ca * Cz));
+        float acc = 0.f;
+        for (int s = 0; s < splits; ++s) acc += __ldcg(partial + (int64_t)s * plane + i);
+        float* d = dw + ((int64_t)j * Ca + c) * taps + tap;
+        *d = accumulate ? (*d + acc) : acc;
+    }
+}
+
+struct ConvTcParams {
+    int Ca, Cz, R, S, pad;
+    int xb, yb, nxb, nyb;        // k-block = xb x yb output positions (xb * yb = 64) of one image
+    int bnc, nv, vgroups;        // B tile = nv horizontal taps x bnc input channels (nv * bnc <= 256)
+    int tiles_c;
+    int splits, kb_per_split, kb_total;
+};
+
+// grid = (tiles_j * tiles_c * R * vgroups, splits).  Warp 0: TMA producer, warp 1: MMA issuer and
+// TMEM owner, warps 2..5: epilogue (one TMEM lane quarter each).
+__global__ void __launch_bounds__(kCThreads, 1)
+conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, float* __restrict__ partial,
+                  int32_t* dev_status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + kCStages * kAStageBytes;
+    ConvTcSmem* ctl = reinterpret_cast<ConvTcSmem*>(sB + kCStages * kBStageBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    int t = blockIdx.x;
+    const int vg = t % p.vgroups; t /= p.vgroups;
+    const int u = t % p.R;        t /= p.R;
+    const int c0 = (t % p.tiles_c) * p.bnc;
+    const int j0 = (t / p.tiles_c) * kBM;
+    const int v0 = vg * p.nv;
+    const int nvt = min(p.nv, p.S - v0);          // horizontal taps stacked in this tile
+    const int ncols = nvt * p.bnc;                // accumulator columns in use
+    const int split = blockIdx.y;
+    const int kb_begin = split * p.kb_per_split;
+    const int kb_end = min(p.kb_total, kb_begin + p.kb_per_split);
+    const int nkb = max(0, kb_end - kb_begin);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kCStages; ++s) {
+            ptx::mbar_init(&ctl->full[s], 1);
+            ptx::mbar_init(&ctl->empty[s], 1);
+        }
+        ptx::mbar_init(&ctl->accum, 1);
+        ctl->abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&maps.dy);
+        for (int i = 0; i < nvt; ++i) ptx::prefetch_tensormap(&maps.x[v0 + i]);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&ctl->tmem_base, kBN);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    volatile int* abort_flag = &ctl->abort_flag;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t stage_bytes = (uint32_t)kAStageBytes + (uint32_t)ncols * 128u;
+            int issued = 0;
+            int xblk = kb_begin % p.nxb;
+            int yblk = (kb_begin / p.nxb) % p.nyb;
+            int n = kb_begin / (p.nxb * p.nyb);
+            for (int i = 0; i < nkb && !*abort_flag; ++i) {
+                const int s = i % kCStages;
+                if (i >= kCStages && !ptx::mbar_wait(&ctl->empty[s], ((i / kCStages) - 1) & 1, kWaitLimit)) {
+                    *abort_flag = 1;
+                    break;
+                }
+                ptx::mbar_arrive_expect_tx(&ctl->full[s], stage_bytes);
+                const int x0 = xblk * p.xb, y0 = yblk * p.yb;
+                tma_load_4d(sA + s * kAStageBytes, &maps.dy, x0, y0, j0, n, &ctl->full[s]);
+                uint8_t* b = sB + s * kBStageBytes;
+                for (int i2 = 0; i2 < nvt; ++i2)
+                    tma_load_4d(b + (size_t)i2 * p.bnc * 128, &maps.x[v0 + i2], x0, y0 + u - p.pad, c0, n, &ctl->full[s]);
+                issued = i + 1;
+                if (++xblk == p.nxb) {
+                    xblk = 0;
+                    if (++yblk == p.nyb) { yblk = 0; ++n; }
+                }
+            }
+            if (*abort_flag) {   // let the copies already in flight land before the CTA exits
+                for (int i = max(0, issued - kCStages); i < issued; ++i)
+                    ptx::mbar_wait(&ctl->full[i % kCStages], (i / kCStages) & 1, kWaitLimit);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = ptx::make_idesc_bf16(kBM, ncols, false, false);   // both operands K-major
+            bool ok = true;
+            for (int i = 0; i < nkb; ++i) {
+                const int s = i % kCStages;
+                if (*abort_flag || !ptx::mbar_wait(&ctl->full[s], (i / kCStages) & 1, kWaitLimit)) {
+                    *abort_flag = 1;
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after();
+                const uint32_t a_addr = ptx::smem_u32(sA + s * kAStageBytes);
+                const uint32_t b_addr = ptx::smem_u32(sB + s * kBStageBytes);
+#pragma unroll
+                for (int kk = 0; kk < kBK / 16; ++kk) {   // 16 k-values = 32 bytes inside the swizzled 128-byte row
+                    const uint64_t ad = ptx::make_smem_desc_sw128(a_addr + kk * 32, 16, 1024);
+                    const uint64_t bd = ptx::make_smem_desc_sw128(b_addr + kk * 32, 16, 1024);
+                    ptx::umma_bf16(tmem_base, ad, bd, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                }
+                ptx::umma_commit(&ctl->empty[s]);
+            }
+            if (ok) ptx::umma_commit(&ctl->accum);
+        }
+    } else if (nkb > 0) {
+        bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
+        ok = __all_sync(kFullMask, ok) && !*abort_flag;
+        if (!ok) {
+            *abort_flag = 1;
+        } else {
+            ptx::tc_fence_after();
+            const int g = warp & 3;
+            const int row = j0 + 32 * g + lane;
+            const int taps = p.R * p.S;
+            const bool vec_ok = (p.Ca & 3) == 0;
+            for (int ch = 0; ch * 32 < ncols; ++ch) {
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
+                ptx::tmem_ld_wait();
+                if (row < p.Cz) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        const int col = ch * 32 + e;       // bnc is a multiple of 16: 4 columns share one tap
+                        if (col < ncols) {
+                            const int vi = col / p.bnc;
+                            const int c = c0 + (col - vi * p.bnc);
+                            const int tap = u * p.S + v0 + vi;
+                            float* dst = partial + (((size_t)split * taps + tap) * p.Cz + row) * p.Ca + c;
+                            if (vec_ok && c + 4 <= p.Ca) {
+                                *reinterpret_cast<float4*>(dst) =
+                                    make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
+                                                __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    if (c + q < p.Ca) dst[q] = __uint_as_float(r[e + q]);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    } else {
+        // an empty split contributes a zero tile
+        const int taps = p.R * p.S;
+        for (int idx = threadIdx.x - 64; idx < kBM * ncols; idx += kCThreads - 64) {
+            const int row = j0 + idx / ncols, col = idx % ncols;
+            const int vi = col / p.bnc;
+            const int c = c0 + (col - vi * p.bnc);
+            if (row < p.Cz && c < p.Ca)
+                partial[(((size_t)split * taps + u * p.S + v0 + vi) * p.Cz + row) * p.Ca + c] = 0.f;
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, kBN);
+    }
+    if (*abort_flag && threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
+}
+
+struct ConvTcPlan {
+    bool ok;
+    int H, W, Ho, Wo;          // geometry the kernel sees (a 1x1 filter flattens each plane into one row)
+    int tiles;
+    ConvTcParams p;
+    size_t dense_stride, partial_off, total_bytes;
+};
+
+ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad, dropit_dtype dtype) {
+    ConvTcPlan pl{};
+    if (dtype != DROPIT_BF16 || stride != 1 || S > kMaxTapsX || pad > kMaxTapsX - 1 || B < 1) return pl;
+    int Ho = H + 2 * pad - R + 1, Wo = W + 2 * pad - S + 1;
+    if (R == 1 && S == 1 && pad == 0) {   // plain GEMM over the flattened plane
+        W = H * W; H = 1; Wo = W; Ho = 1;
+    }
+    if (Wo > W || (W & 7) || (Wo & 7)) return pl;   // TMA strides are multiples of 16 bytes
+    ConvTcParams& p = pl.p;
+    p.Ca = Ca; p.Cz = Cz; p.R = R; p.S = S; p.pad = pad;
+    // One k-block = 64 consecutive pixels of one image row, so a tile row is exactly one 128-byte
+    // swizzle row.  (Boxes with a narrower inner extent and several image rows are not used: their
+    // shared-memory footprint under the 128-byte swizzle is not the dense one.)
+    p.xb = 64; p.yb = 1;
+    p.nxb = (Wo + p.xb - 1) / p.xb;
+    p.nyb = (Ho + p.yb - 1) / p.yb;
+    const int64_t kb_total = (int64_t)B * p.nxb * p.nyb;
+    if (kb_total >= (1ll << 30)) return pl;
+    p.kb_total = (int)kb_total;
+    p.bnc = Ca >= kBN ? kBN : (Ca + 15) / 16 * 16;
+    p.nv = kBN / p.bnc < S ? kBN / p.bnc : S;
+    if (p.nv < 1) p.nv = 1;
+    p.vgroups = (S + p.nv - 1) / p.nv;
+    p.tiles_c = (Ca + p.bnc - 1) / p.bnc;
+    const int64_t tiles = (int64_t)((Cz + kBM - 1) / kBM) * p.tiles_c * R * p.vgroups;
+    if (tiles > (1ll << 30)) return pl;
+    pl.tiles = (int)tiles;
+    int splits = sm_count() / pl.tiles;
+    if (splits < 1) splits = 1;
+    if (splits > p.kb_total) splits = p.kb_total;
+    p.kb_per_split = (p.kb_total + splits - 1) / splits;
+    p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+    if (p.splits > 65535) return pl;
+    pl.H = H; pl.W = W; pl.Ho = Ho; pl.Wo = Wo;
+    pl.dense_stride = align_up((size_t)B * Ca * H * W * 2, 256);
+    pl.partial_off = pl.dense_stride * S;
+    pl.total_bytes = pl.partial_off + align_up((size_t)p.splits * R * S * Cz * Ca * 4, 256);
+    pl.ok = true;
+    return pl;
+}
+
+}  // namespace
+
+// 0 when the tensor-core path does not take this shape.
+size_t conv_tc_workspace_bytes(int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad,
+                               dropit_dtype dtype) {
+    const ConvTcPlan pl = make_conv_tc_plan(B, Ca, H, W, Cz, R, S, stride, pad, dtype);
+    return pl.ok ? pl.total_bytes : 0;
+}
+
+// Caller has validated pointers, sizes and alignment, and B >= 1, k >= 1.
+dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, const uint32_t* offsets, int B, int Ca,
+                          int H, int W, int Cz, int R, int S, int stride, int pad, int64_t k, dropit_format format,
+                          float* dw, int accumulate, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                          cudaStream_t stream) {
+    const ConvTcPlan pl = make_conv_tc_plan(B, Ca, H, W, Cz, R, S, stride, pad, DROPIT_BF16);
+    if (!pl.ok) return DROPIT_ERR_UNSUPPORTED;
+    if (workspace_bytes < pl.total_bytes) return DROPIT_ERR_WORKSPACE;
+    unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
+    const int64_t n = (int64_t)B * Ca * H * W;
+    // the unshifted copy lives in slot `pad`, so slot v always holds the rows shifted by v - pad
+    void* dense0 = ws + pl.dense_stride * pad;
+    dropit_status st = decompress_dispatch(values, meta, offsets, n, k, DROPIT_BF16, format, dense0, stream);
+    if (st != DROPIT_OK) return st;
+    if (S > 1) {
+        ShiftDst dst{};
+        for (int v = 0; v < S; ++v)
+            if (v != pad) dst.out[v - pad + kMaxTapsX - 1] = reinterpret_cast<uint4*>(ws + pl.dense_stride * v);
+        const int64_t groups = n / 8;
+        int64_t blocks = (groups + 255) / 256;
+        if (blocks > (int64_t)sm_count() * 16) blocks = (int64_t)sm_count() * 16;
+        shift_copies_kernel<<<(unsigned)blocks, 256, 0, stream>>>(reinterpret_cast<const uint4*>(dense0), dst, groups,
+                                                                 pl.W / 8);
+        st = check_launch();
+        if (st != DROPIT_OK) return st;
+    }
+    ConvMaps maps;
+    if (!make_map_nchw(&maps.dy, dy, B, Cz, pl.Ho, pl.Wo, pl.p.xb, pl.p.yb, kBM)) return DROPIT_ERR_CUDA;
+    for (int v = 0; v < kMaxTapsX; ++v) {
+        const int slot = v < S ? v : pad;
+        if (!make_map_nchw(&maps.x[v], ws + pl.dense_stride * slot, B, Ca, pl.H, pl.W, pl.p.xb, pl.p.yb, pl.p.bnc))
+            return DROPIT_ERR_CUDA;
+    }
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(conv_wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kConvTcSmemBytes) != cudaSuccess)
+            return DROPIT_ERR_CUDA;
+        attr_set = true;
+    }
+    float* partial = reinterpret_cast<float*>(ws + pl.partial_off);
+    dim3 grid(pl.tiles, pl.p.splits);
+    conv_wg_tc_kernel<<<grid, kCThreads, kConvTcSmemBytes, stream>>>(maps, pl.p, partial, dev_status);
+    st = check_launch();
+    if (st != DROPIT_OK) return st;
+    const int64_t count = (int64_t)R * S * Cz * Ca;
+    int64_t blocks = (count + 255) / 256;
+    if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
+    conv_tc_reduce_kernel<<<(unsigned)blocks, 256, 0, stream>>>(partial, pl.p.splits, Cz, Ca, R * S, dw, accumulate);
+    return check_launch();
+}
+
+}  // namespace dropit

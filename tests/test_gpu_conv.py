@@ -22,6 +22,16 @@ SMALL = [
     di.small_conv(2, 8, 10, 10, 8, 3, 2, 1, 0, "bf16", 0.0),         # gamma = 0, no padding, non-square filter
     di.small_conv(2, 8, 10, 10, 8, 3, 3, 1, 1, "bf16", 1.0),         # gamma = 1
     di.small_conv(70, 8, 6, 6, 8, 3, 3, 1, 1, "bf16", 0.8),          # more images than splits
+    # shapes the tensor-core path takes (bf16, stride 1, rows a multiple of 8 pixels)
+    di.small_conv(2, 16, 16, 16, 32, 3, 3, 1, 1, "bf16", 0.8),       # k-block = 4 rows x 16 pixels
+    di.small_conv(2, 24, 8, 8, 40, 3, 3, 1, 1, "bf16", 0.8),         # k-block = 8 x 8, three taps stacked in N
+    di.small_conv(3, 130, 24, 32, 200, 3, 3, 1, 1, "bf16", 0.8),     # two row tiles, ragged channel tile
+    di.small_conv(2, 300, 16, 16, 20, 1, 1, 1, 0, "bf16", 0.8),      # 1x1: flattened plane, two channel tiles
+    di.small_conv(2, 8, 16, 24, 8, 5, 5, 1, 2, "bf16", 0.5),         # 25 taps, five stacked
+    di.small_conv(2, 8, 12, 16, 8, 3, 1, 1, 0, "bf16", 0.8),         # no padding: Ho < H
+    di.small_conv(1, 16, 4, 72, 16, 3, 3, 1, 1, "bf16", 0.8),        # rows wider than one k-block
+    di.small_conv(2, 3, 16, 16, 8, 7, 7, 1, 3, "bf16", 0.5),         # 7x7 on 3 channels
+    di.small_conv(150, 8, 8, 8, 8, 3, 3, 1, 1, "bf16", 0.8),         # more k-blocks than splits, uneven
     di.small_conv(4, 64, 56, 56, 64, 3, 3, 1, 1, "bf16", 0.8),       # the ResNet stage-1 3x3 shape, 4 images
     di.small_conv(4, 256, 56, 56, 64, 1, 1, 1, 0, "bf16", 0.8),      # the ResNet stage-1 1x1 shape, 4 images
 ]
