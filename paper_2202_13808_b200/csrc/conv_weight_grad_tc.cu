@@ -187,7 +187,7 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
             int n = kb_begin / (p.nxb * p.nyb);
             for (int i = 0; i < nkb && !*abort_flag; ++i) {
                 const int s = i % kCStages;
-                if (i >= kCStages && !ptx::mbar_wait(&ctl->empty[s], ((i / kCStages) - 1) & 1, kWaitLimit)) {
+                if (i >= kCStages && !ptx::mbar_wait_spin(&ctl->empty[s], ((i / kCStages) - 1) & 1, kWaitLimit)) {
                     *abort_flag = 1;
                     break;
                 }
@@ -214,7 +214,7 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
             bool ok = true;
             for (int i = 0; i < nkb; ++i) {
                 const int s = i % kCStages;
-                if (*abort_flag || !ptx::mbar_wait(&ctl->full[s], (i / kCStages) & 1, kWaitLimit)) {
+                if (*abort_flag || !ptx::mbar_wait_spin(&ctl->full[s], (i / kCStages) & 1, kWaitLimit)) {
                     *abort_flag = 1;
                     ok = false;
                     break;
@@ -378,11 +378,10 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
     }
     ConvMaps maps;
     if (!make_map_nchw(&maps.dy, dy, B, Cz, pl.Ho, pl.Wo, pl.p.xb, pl.p.yb, kBM)) return DROPIT_ERR_CUDA;
-    for (int v = 0; v < kMaxTapsX; ++v) {
-        const int slot = v < S ? v : pad;
-        if (!make_map_nchw(&maps.x[v], ws + pl.dense_stride * slot, B, Ca, pl.H, pl.W, pl.p.xb, pl.p.yb, pl.p.bnc))
+    for (int v = 0; v < S; ++v)
+        if (!make_map_nchw(&maps.x[v], ws + pl.dense_stride * v, B, Ca, pl.H, pl.W, pl.p.xb, pl.p.yb, pl.p.bnc))
             return DROPIT_ERR_CUDA;
-    }
+    for (int v = S; v < kMaxTapsX; ++v) maps.x[v] = maps.x[0];   // never read; keeps the parameter defined
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(conv_wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -43,6 +43,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
     }
     return false;
 }
+// Bounded wait without back-off, for the single thread that issues TMA copies or MMAs: try_wait already
+// suspends the thread for a hardware-chosen time, and a sleep here would add to every pipeline hand-over.
+__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
 // Whole-warp bounded wait: lane 0 polls (an mbarrier poll costs on the order of 100 cycles), the
 // warp-level exchange of the result orders the other lanes' later reads after lane 0's acquire.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, uint32_t limit) {

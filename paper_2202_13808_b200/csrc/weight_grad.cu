@@ -66,7 +66,7 @@ static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype
         p.splits = 1;
     }
     p.counters_off = 0;
-    p.counters_bytes = align_up((size_t)p.tiles_m * p.tiles_n * 4, 256);
+    p.counters_bytes = align_up((size_t)p.tiles_m * p.tiles_n * 8, 256);   // per tile: tickets drawn, partial planes published
     p.dense_off = p.counters_off + p.counters_bytes;
     p.dense_bytes = p.fused ? 0 : align_up((size_t)M * Ca * es, 256);
     p.partial_off = p.dense_off + p.dense_bytes;
@@ -116,9 +116,94 @@ struct TcSmem {
     uint64_t accum;
     uint32_t tmem_base;
     int abort_flag;
-    int is_last;
+    int finisher;     // this CTA drew the last ticket of its tile: it adds the partial tiles and writes dW
 };
+constexpr int kEpiRowFloats = 36;                          // staging row pitch: 32 columns + 4 (bank spread, 16-byte rows)
+constexpr int kEpiWarpFloats = 32 * kEpiRowFloats;         // one warp's 32 x 32 chunk
+constexpr int kEpiSpinLimit = 1 << 20;
 constexpr size_t kTcSmemBytes = 1024 + (size_t)kStages * (kAStageBytes + kBStageBytes) + sizeof(TcSmem);
+
+// Epilogue of one 128 x 256 accumulator tile, run by the four warps that own the TMEM lane quarters.
+// Each 32 x 32 chunk goes TMEM -> registers -> shared memory (row pitch 36 floats) and leaves as full
+// 128-byte row segments.  A CTA that is not its tile's finisher stores the chunk into its split's
+// partial plane.  The finisher adds the planes in split order, taking its own term from the chunk, so
+// the sum does not depend on which split finishes last, and writes dW.
+__device__ __forceinline__ void epilogue_tile_staged(uint32_t tmem_base, float* stage, int g, int lane, int j0, int c0,
+                                                     int Ca, int Cz, int split, int splits, bool finisher,
+                                                     float* __restrict__ dw, int accumulate,
+                                                     float* __restrict__ partial) {
+    const size_t plane = (size_t)Cz * Ca;
+    const int rr0 = lane >> 3, q = lane & 7;
+#pragma unroll 1
+    for (int ch = 0; ch < kBN / 32; ++ch) {
+        const int col = c0 + ch * 32 + 4 * q;
+        const bool col_ok = col < Ca;            // Ca is a multiple of 8
+        size_t off[8];
+        bool ok[8];
+        float4 acc[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int row = j0 + 32 * g + it * 4 + rr0;
+            ok[it] = col_ok && row < Cz;
+            off[it] = ok[it] ? (size_t)row * Ca + col : 0;
+            acc[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (finisher && accumulate) {
+#pragma unroll
+            for (int it = 0; it < 8; ++it)
+                if (ok[it]) acc[it] = *reinterpret_cast<const float4*>(dw + off[it]);
+        }
+        float4 other[8];
+        if (finisher && splits == 2) {           // the common case: the other plane's loads fly during the TMEM read
+#pragma unroll
+            for (int it = 0; it < 8; ++it)
+                other[it] = ok[it] ? __ldcg(reinterpret_cast<const float4*>(partial + (size_t)(1 - split) * plane + off[it]))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<float4*>(stage + lane * kEpiRowFloats + e) =
+                make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
+                            __uint_as_float(r[e + 3]));
+        __syncwarp();
+        float4 own[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it)
+            own[it] = *reinterpret_cast<const float4*>(stage + (it * 4 + rr0) * kEpiRowFloats + 4 * q);
+        __syncwarp();
+        if (!finisher) {
+#pragma unroll
+            for (int it = 0; it < 8; ++it)
+                if (ok[it]) *reinterpret_cast<float4*>(partial + (size_t)split * plane + off[it]) = own[it];
+            continue;
+        }
+        for (int s = 0; s < splits; ++s) {       // fixed order over the splits
+            float4 v[8];
+            if (s == split) {
+#pragma unroll
+                for (int it = 0; it < 8; ++it) v[it] = own[it];
+            } else if (splits == 2) {
+#pragma unroll
+                for (int it = 0; it < 8; ++it) v[it] = other[it];
+            } else {
+#pragma unroll
+                for (int it = 0; it < 8; ++it)
+                    v[it] = ok[it] ? __ldcg(reinterpret_cast<const float4*>(partial + (size_t)s * plane + off[it]))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                acc[it].x += v[it].x; acc[it].y += v[it].y; acc[it].z += v[it].z; acc[it].w += v[it].w;
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it)
+            if (ok[it]) *reinterpret_cast<float4*>(dw + off[it]) = acc[it];
+    }
+}
 
 __global__ void __launch_bounds__(kTcThreads, 1)
 wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, int Ca, int Cz,
@@ -147,7 +232,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         }
         ptx::mbar_init(&ctl->accum, 1);
         ctl->abort_flag = 0;
-        ctl->is_last = 0;
+        ctl->finisher = 1;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&map_dy);
         ptx::prefetch_tensormap(&map_x);
@@ -168,7 +253,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
             int issued = 0;
             for (int i = 0; i < nkb && !*abort_flag; ++i) {
                 const int s = i % kStages;
-                if (i >= kStages && !ptx::mbar_wait(&ctl->empty[s], ((i / kStages) - 1) & 1, kWaitLimit)) {
+                if (i >= kStages && !ptx::mbar_wait_spin(&ctl->empty[s], ((i / kStages) - 1) & 1, kWaitLimit)) {
                     *abort_flag = 1;
                     break;
                 }
@@ -195,7 +280,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
             bool ok = true;
             for (int i = 0; i < nkb; ++i) {
                 const int s = i % kStages;
-                if (*abort_flag || !ptx::mbar_wait(&ctl->full[s], (i / kStages) & 1, kWaitLimit)) {
+                if (*abort_flag || !ptx::mbar_wait_spin(&ctl->full[s], (i / kStages) & 1, kWaitLimit)) {
                     *abort_flag = 1;
                     ok = false;
                     break;
@@ -217,11 +302,38 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         // ---------------- epilogue: TMEM -> global ----------------
         bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
         ok = __all_sync(kFullMask, ok) && !*abort_flag;
-        if (!ok) {
-            *abort_flag = 1;
-        } else {
+        if (!ok) *abort_flag = 1;
+        // The accumulator is final, so every MMA has read its operands and every TMA copy has landed:
+        // the pipeline buffers are free and serve as the staging area.
+        uint32_t* tickets = counters + tile;
+        uint32_t* done = counters + gridDim.x + tile;
+        if (splits > 1) {
+            if (threadIdx.x == 64) ctl->finisher = (atomicAdd(tickets, 1u) == (uint32_t)splits - 1) ? 1 : 0;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        const bool finisher = ctl->finisher != 0;
+        if (finisher && splits > 1) {
+            // the other splits of this tile have drawn their tickets, so they are running their epilogues
+            if (threadIdx.x == 64) {
+                int spins = 0;
+                while (*reinterpret_cast<volatile uint32_t*>(done) < (uint32_t)splits - 1 && !*abort_flag) {
+                    if (++spins > kEpiSpinLimit) { *abort_flag = 1; break; }
+                    __nanosleep(64);
+                }
+                __threadfence();
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        if (!*abort_flag) {
             ptx::tc_fence_after();
-            epilogue_store_tile(tmem_base, warp, lane, j0, c0, Ca, Cz, split, splits, dw, accumulate, partial);
+            float* stage = reinterpret_cast<float*>(smem) + (warp - 2) * kEpiWarpFloats;
+            epilogue_tile_staged(tmem_base, stage, warp & 3, lane, j0, c0, Ca, Cz, split, splits, finisher, dw,
+                                 accumulate, partial);
+        }
+        if (!finisher) {   // publish the partial plane (also after an abort, so that the finisher's wait ends)
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64) atomicAdd(done, 1u);
         }
     }
 
@@ -231,13 +343,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kBN);
     }
-    if (*abort_flag) {
-        if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
-        return;
-    }
-    if (splits == 1) return;
-
-    split_reduce_tile(tile, j0, c0, Ca, Cz, splits, dw, accumulate, partial, counters, &ctl->is_last);
+    if (*abort_flag && threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
 }
 
 // ---------------------------------------------------------------------------------------------
