@@ -5,48 +5,64 @@ namespace dropit {
 
 unsigned long long g_launch_count = 0;
 
-// One thread per 16-byte output vector.  The number of retained elements before the vector is
-// the chunk's table entry plus the mask bits of the chunk that precede it.
+// A warp inflates 1024 consecutive elements (32 mask words, 8 chunks) per step: lane l owns word l.
+// Its first retained element sits at the chunk's table entry plus the population of the chunk's
+// earlier words.  The lane drops its retained values into a zeroed shared-memory image of the 1024
+// elements (work proportional to the number of retained values, not to the dense size), and the warp
+// then streams the image out as 512-byte store instructions.
+constexpr int kDecompWarps = 8;
+
 template <typename Tr>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(32 * kDecompWarps)
 decompress_bitmask_kernel(const typename Tr::elem_t* __restrict__ values, const uint32_t* __restrict__ mask,
                           const uint32_t* __restrict__ offsets, int64_t n, typename Tr::elem_t* __restrict__ out) {
     using elem_t = typename Tr::elem_t;
-    constexpr int G = Tr::kVecElems;
-    const int64_t nvec = (n + G - 1) / G;
+    constexpr int G = Tr::kVecElems;                 // elements per 16-byte vector
+    constexpr int kPitch = 32 + G;                   // image row = one mask word; one spare vector spreads the banks
+    constexpr int kVecPerRow = 32 / G;
+    __shared__ __align__(16) elem_t image[kDecompWarps][32 * kPitch];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    elem_t* img = image[warp];
     const int64_t nwords = (n + 31) / 32;
-    for (int64_t vi = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; vi < nvec; vi += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t e0 = vi * G;
-        const int64_t chunk = e0 / DROPIT_CHUNK;
-        const int b = (int)(e0 % DROPIT_CHUNK);
-        const int64_t w0 = chunk * (DROPIT_CHUNK / 32);
-        uint32_t pos = offsets[chunk];
-        const int wi = b >> 5;
-        for (int w = 0; w < wi; ++w) pos += __popc(mask[w0 + w]);
-        const uint32_t word = (w0 + wi < nwords) ? mask[w0 + wi] : 0u;
-        const int sh = b & 31;
-        pos += __popc(word & ((1u << sh) - 1u));
-        const uint32_t bits = (word >> sh) & ((1u << G) - 1u);
-        elem_t r[G];
+    const int64_t ntiles = (nwords + 31) / 32;
+    for (int64_t t = (int64_t)blockIdx.x * kDecompWarps + warp; t < ntiles; t += (int64_t)gridDim.x * kDecompWarps) {
+        const int64_t w = t * 32 + lane;
+        uint32_t word = (w < nwords) ? __ldg(mask + w) : 0u;
+        const int64_t e_word = w * 32;
+        if (e_word + 32 > n) word = (e_word < n) ? (word & ((1u << (int)(n - e_word)) - 1u)) : 0u;
+        const uint32_t cnt = __popc(word);
+        uint32_t incl = cnt;                         // inclusive count over the lanes of this chunk (4 words)
+        uint32_t up = __shfl_up_sync(kFullMask, incl, 1);
+        if ((lane & 3) >= 1) incl += up;
+        up = __shfl_up_sync(kFullMask, incl, 2);
+        if ((lane & 3) >= 2) incl += up;
+        uint32_t pos = (w < nwords) ? __ldg(offsets + (w >> 2)) : 0u;
+        pos += incl - cnt;
+        const uint4 zero = make_uint4(0, 0, 0, 0);
 #pragma unroll
-        for (int e = 0; e < G; ++e) {
-            r[e] = 0;
-            if ((bits >> e) & 1u) r[e] = values[pos++];
+        for (int i = 0; i < kPitch / G; ++i) reinterpret_cast<uint4*>(img)[i * 32 + lane] = zero;
+        __syncwarp();
+        while (word) {
+            const int b = __ffs(word) - 1;
+            word &= word - 1;
+            img[lane * kPitch + b] = values[pos++];
         }
-        if (e0 + G <= n) {
-            uint4 o;
-            if constexpr (G == 8) {
-                o.x = r[0] | ((uint32_t)r[1] << 16);
-                o.y = r[2] | ((uint32_t)r[3] << 16);
-                o.z = r[4] | ((uint32_t)r[5] << 16);
-                o.w = r[6] | ((uint32_t)r[7] << 16);
-            } else {
-                o = make_uint4(r[0], r[1], r[2], r[3]);
+        __syncwarp();
+        const int64_t e_tile = t * 1024;
+#pragma unroll
+        for (int i = 0; i < kVecPerRow; ++i) {
+            const int v = i * 32 + lane;             // vector of the tile, in output order
+            const int row = v / kVecPerRow, col = v % kVecPerRow;
+            const int64_t e0 = e_tile + (int64_t)v * G;
+            const uint4 o = *reinterpret_cast<const uint4*>(img + row * kPitch + col * G);
+            if (e0 + G <= n) {
+                *reinterpret_cast<uint4*>(out + e0) = o;
+            } else if (e0 < n) {
+                const elem_t* src = img + row * kPitch + col * G;
+                for (int e = 0; e0 + e < n; ++e) out[e0 + e] = src[e];
             }
-            reinterpret_cast<uint4*>(out)[vi] = o;
-        } else {
-            for (int e = 0; e0 + e < n; ++e) out[e0 + e] = r[e];
         }
+        __syncwarp();
     }
 }
 
@@ -66,10 +82,10 @@ static dropit_status run_decompress(const void* values, const void* meta, const 
     using elem_t = typename Tr::elem_t;
     const int64_t cap = (int64_t)sm_count() * 16;
     if (format == DROPIT_FMT_BITMASK) {
-        const int64_t nvec = (n + Tr::kVecElems - 1) / Tr::kVecElems;
-        int64_t blocks = (nvec + 255) / 256;   // one vector per thread: short threads, many in flight
-        if (blocks > 0x7FFFFFFF) blocks = 0x7FFFFFFF;
-        decompress_bitmask_kernel<Tr><<<(unsigned)blocks, 256, 0, stream>>>(
+        const int64_t ntiles = (n + 1023) / 1024;       // one warp step each
+        int64_t blocks = (ntiles + kDecompWarps - 1) / kDecompWarps;
+        if (blocks > cap * 4) blocks = cap * 4;
+        decompress_bitmask_kernel<Tr><<<(unsigned)blocks, 32 * kDecompWarps, 0, stream>>>(
             reinterpret_cast<const elem_t*>(values), reinterpret_cast<const uint32_t*>(meta), offsets, n,
             reinterpret_cast<elem_t*>(out));
         return check_launch();

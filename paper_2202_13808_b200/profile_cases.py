@@ -27,7 +27,7 @@ CASES = {c.name: c for c in (di.SINGLE_LINEAR_F32, di.VITB_FC1, di.VITB_FC2, di.
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["compress", "weight_grad", "conv_weight_grad"])
+    ap.add_argument("op", choices=["compress", "decompress", "weight_grad", "conv_weight_grad"])
     ap.add_argument("case", choices=sorted(CASES))
     ap.add_argument("--gamma", type=float, default=None)
     ap.add_argument("--format", default="bitmask", choices=["bitmask", "index32"])
@@ -37,7 +37,7 @@ def main():
     gamma = case.gamma if args.gamma is None else args.gamma
     dev = torch.device("cuda:0")
     x = di.make_x(case).to(dev)
-    dy = di.make_dy(case).to(dev) if args.op != "compress" else None
+    dy = di.make_dy(case).to(dev) if args.op in ("weight_grad", "conv_weight_grad") else None
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     cache = dropit.dropit_compress(x, gamma, args.format)
     for r in range(args.reps):
@@ -47,6 +47,8 @@ def main():
         e0.record()
         if args.op == "compress":
             cache = dropit.dropit_compress(x, gamma, args.format)
+        elif args.op == "decompress":
+            dropit.dropit_decompress(cache)
         elif args.op == "weight_grad":
             dropit.dropit_weight_grad(dy, cache)
         else:
