@@ -33,6 +33,7 @@ constexpr int kTcThreads = 192;
 struct WgPlan {
     bool tensor_core;
     bool fused;               // expand the bitmask cache inside the GEMM (no dense scratch)
+    bool cluster;             // the splits of a tile form a thread-block cluster and add up through shared memory
     int tiles_m, tiles_n, splits, kb_total, kb_per_split;
     size_t counters_off, counters_bytes;
     size_t dense_off, dense_bytes;
@@ -60,6 +61,7 @@ static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype
         if (splits > p.kb_total) splits = p.kb_total;
         p.kb_per_split = (p.kb_total + splits - 1) / splits;
         p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;   // every split owns >= 1 block
+        p.cluster = !p.fused && (p.splits == 2 || p.splits == 4);
     } else {
         p.tiles_m = (int)((Cz + 63) / 64);
         p.tiles_n = (int)((Ca + 63) / 64);
@@ -70,7 +72,7 @@ static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype
     p.dense_off = p.counters_off + p.counters_bytes;
     p.dense_bytes = p.fused ? 0 : align_up((size_t)M * Ca * es, 256);
     p.partial_off = p.dense_off + p.dense_bytes;
-    p.partial_bytes = (p.splits > 1) ? align_up((size_t)p.splits * Cz * Ca * 4, 256) : 0;
+    p.partial_bytes = (p.splits > 1 && !p.cluster) ? align_up((size_t)p.splits * Cz * Ca * 4, 256) : 0;
     p.total_bytes = p.partial_off + p.partial_bytes;
     if (p.total_bytes == 0) p.total_bytes = 256;
     return p;
@@ -121,6 +123,8 @@ struct TcSmem {
 constexpr int kEpiRowFloats = 36;                          // staging row pitch: 32 columns + 4 (bank spread, 16-byte rows)
 constexpr int kEpiWarpFloats = 32 * kEpiRowFloats;         // one warp's 32 x 32 chunk
 constexpr int kEpiSpinLimit = 1 << 20;
+constexpr int kXchgRowFloats = kBN + 4;                    // exchange row pitch: lanes of a warp (rows) hit distinct banks
+constexpr int kXchgMaxBytes = 3 * 32 * kXchgRowFloats * 4; // 4 splits: three peers send 32 rows each (2 splits: one sends 64)
 constexpr size_t kTcSmemBytes = 1024 + (size_t)kStages * (kAStageBytes + kBStageBytes) + sizeof(TcSmem);
 
 // Epilogue of one 128 x 256 accumulator tile, run by the four warps that own the TMEM lane quarters.
@@ -205,11 +209,90 @@ __device__ __forceinline__ void epilogue_tile_staged(uint32_t tmem_base, float* 
     }
 }
 
+// Split reduction inside a thread-block cluster (2 or 4 splits of one tile are the CTAs of one cluster).
+// The tile's four 32-row quarters are shared out among the CTAs; every CTA sends the quarters it does
+// not own from TMEM into the owner's shared memory, the owner adds the terms in split order (its own
+// from TMEM) and writes dW.  Called by the four epilogue warps between the cluster barriers.
+__device__ __forceinline__ int quarter_owner(int g, int splits) { return g * splits / 4; }
+
+__device__ __forceinline__ void cluster_send_quarter(uint32_t tmem_base, uint8_t* xchg, int g, int lane, int rank,
+                                                     int splits) {
+    const int owner = quarter_owner(g, splits);
+    const int slot = rank < owner ? rank : rank - 1;                 // the owner keeps no slot for itself
+    const int rows_owned = 128 / splits;
+    const int row_local = (g - owner * (4 / splits)) * 32 + lane;
+    const uint32_t local = ptx::smem_u32(xchg) + (uint32_t)((slot * rows_owned + row_local) * kXchgRowFloats) * 4u;
+    const uint32_t remote = ptx::map_shared_to_cta(local, (uint32_t)owner);
+#pragma unroll 1
+    for (int ch = 0; ch < kBN / 32; ++ch) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; e += 4)
+            ptx::st_cluster_v4(remote + (uint32_t)(ch * 32 + e) * 4u, __uint_as_float(r[e]), __uint_as_float(r[e + 1]),
+                               __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+    }
+}
+
+__device__ __forceinline__ void cluster_finish_quarter(uint32_t tmem_base, const uint8_t* xchg, float* stage, int g,
+                                                       int lane, int rank, int splits, int j0, int c0, int Ca, int Cz,
+                                                       float* __restrict__ dw, int accumulate) {
+    const int rows_owned = 128 / splits;
+    const int row_local = (g - rank * (4 / splits)) * 32 + lane;
+    const float* mine = reinterpret_cast<const float*>(xchg) + (size_t)row_local * kXchgRowFloats;
+    const int rr0 = lane >> 3, q = lane & 7;
+#pragma unroll 1
+    for (int ch = 0; ch < kBN / 32; ++ch) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
+        ptx::tmem_ld_wait();
+        float acc[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+        for (int s = 0; s < splits; ++s) {                            // fixed order over the splits
+            if (s == rank) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(r[e]);
+            } else {
+                const int slot = s < rank ? s : s - 1;
+                const float* src = mine + (size_t)slot * rows_owned * kXchgRowFloats + ch * 32;
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 v = *reinterpret_cast<const float4*>(src + e);
+                    acc[e] += v.x; acc[e + 1] += v.y; acc[e + 2] += v.z; acc[e + 3] += v.w;
+                }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<float4*>(stage + lane * kEpiRowFloats + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
+        __syncwarp();
+        const int col = c0 + ch * 32 + 4 * q;
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int row = j0 + 32 * g + it * 4 + rr0;
+            if (col < Ca && row < Cz) {
+                float4 v = *reinterpret_cast<const float4*>(stage + (it * 4 + rr0) * kEpiRowFloats + 4 * q);
+                float* dst = dw + (size_t)row * Ca + col;
+                if (accumulate) {
+                    const float4 o = *reinterpret_cast<const float4*>(dst);
+                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                }
+                *reinterpret_cast<float4*>(dst) = v;
+            }
+        }
+        __syncwarp();
+    }
+}
+
 __global__ void __launch_bounds__(kTcThreads, 1)
 wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, int Ca, int Cz,
              int tiles_n, int splits, int kb_per_split, int kb_total, float* __restrict__ dw, int accumulate,
-             float* __restrict__ partial, uint32_t* counters, int32_t* dev_status) {
+             float* __restrict__ partial, uint32_t* counters, int32_t* dev_status, int cluster_mode) {
     extern __shared__ uint8_t smem_raw[];
+    // The dynamic window starts at the same offset in every CTA of the kernel, so this rounding gives
+    // the same offsets in both CTAs of a cluster (the exchange below maps addresses between them).
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
     uint8_t* sB = smem + kStages * kAStageBytes;
@@ -218,7 +301,8 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int tile = blockIdx.x;
-    const int split = blockIdx.y;
+    // cluster mode: the cluster is (1, splits, 1), its CTA rank is the split
+    const int split = cluster_mode ? (int)ptx::cluster_ctarank() : (int)blockIdx.y;
     const int j0 = (tile / tiles_n) * kBM;
     const int c0 = (tile % tiles_n) * kBN;
     const int kb_begin = split * kb_per_split;
@@ -303,6 +387,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
         ok = __all_sync(kFullMask, ok) && !*abort_flag;
         if (!ok) *abort_flag = 1;
+        if (!cluster_mode) {
         // The accumulator is final, so every MMA has read its operands and every TMA copy has landed:
         // the pipeline buffers are free and serve as the staging area.
         uint32_t* tickets = counters + tile;
@@ -335,6 +420,25 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (threadIdx.x == 64) atomicAdd(done, 1u);
         }
+        }   // ticket path
+    }
+
+    if (cluster_mode) {
+        // All roles are done here: the accumulator is final and the pipeline buffers of this CTA are free.
+        // Every thread of the cluster takes part in the two barriers, whatever happened before.
+        uint8_t* xchg = smem;                                              // receive area, <= kXchgMaxBytes
+        float* stage = reinterpret_cast<float*>(smem + kXchgMaxBytes) + (warp >= 2 ? (warp - 2) * kEpiWarpFloats : 0);
+        __syncwarp();
+        ptx::cluster_sync_all();                                           // every CTA's buffers are free
+        const int g = warp & 3;
+        if (warp >= 2 && !*abort_flag) {
+            ptx::tc_fence_after();
+            if (quarter_owner(g, splits) != split) cluster_send_quarter(tmem_base, xchg, g, lane, split, splits);
+        }
+        __syncwarp();
+        ptx::cluster_sync_all();                                           // every quarter has been delivered
+        if (warp >= 2 && !*abort_flag && quarter_owner(g, splits) == split)
+            cluster_finish_quarter(tmem_base, xchg, stage, g, lane, split, splits, j0, c0, Ca, Cz, dw, accumulate);
     }
 
     ptx::tc_fence_before();
@@ -474,7 +578,7 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     if (!make_map_2d_bf16(&map_dy, dy, M, Cz) || !make_map_2d_bf16(&map_x, dense, M, Ca)) return DROPIT_ERR_CUDA;
     uint32_t* counters = reinterpret_cast<uint32_t*>(ws + plan.counters_off);
     float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
-    if (plan.splits > 1 && cudaMemsetAsync(counters, 0, plan.counters_bytes, stream) != cudaSuccess)
+    if (plan.splits > 1 && !plan.cluster && cudaMemsetAsync(counters, 0, plan.counters_bytes, stream) != cudaSuccess)
         return DROPIT_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
@@ -484,9 +588,26 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
         attr_set = true;
     }
     dim3 grid(plan.tiles_m * plan.tiles_n, plan.splits);
-    wg_tc_kernel<<<grid, kTcThreads, kTcSmemBytes, stream>>>(map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n,
-                                                            plan.splits, plan.kb_per_split, plan.kb_total, dw,
-                                                            accumulate, partial, counters, dev_status);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = kTcSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    if (plan.cluster) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1;
+        attr[0].val.clusterDim.y = (unsigned)plan.splits;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    if (cudaLaunchKernelEx(&cfg, wg_tc_kernel, map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n, plan.splits,
+                           plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status,
+                           plan.cluster ? 1 : 0) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DROPIT_ERR_CUDA;
+    }
     return check_launch();
 }
 
