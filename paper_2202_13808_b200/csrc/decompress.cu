@@ -1,5 +1,6 @@
 // R(a-hat): inflate the sparse cache to a dense tensor, dropped positions = +0 (Sec. 3.2).
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace dropit {
 
@@ -21,6 +22,7 @@ decompress_bitmask_kernel(const typename Tr::elem_t* __restrict__ values, const 
     constexpr int kPitch = 32 + G;                   // image row = one mask word; one spare vector spreads the banks
     constexpr int kVecPerRow = 32 / G;
     __shared__ __align__(16) elem_t image[kDecompWarps][32 * kPitch];
+    ptx::launch_dependents();   // a weight-gradient kernel behind this one may set itself up meanwhile
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     elem_t* img = image[warp];
     const int64_t nwords = (n + 31) / 32;
@@ -70,6 +72,7 @@ template <typename Tr>
 __global__ void __launch_bounds__(256)
 scatter_index32_kernel(const typename Tr::elem_t* __restrict__ values, const int32_t* __restrict__ idx, int64_t k,
                        int64_t n, typename Tr::elem_t* __restrict__ out) {
+    ptx::launch_dependents();
     for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < k; r += (int64_t)gridDim.x * blockDim.x) {
         const int64_t i = idx[r];
         if (i >= 0 && i < n) out[i] = values[r];

@@ -77,6 +77,14 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 
+// ---- programmatic dependent launch ----
+// launch_dependents: the next kernel of the stream, if it was launched with programmatic stream
+// serialization, may start once every CTA of this grid has executed this (or exited).
+// grid_dependency_wait: blocks until the preceding grid has completed and its writes are visible; a
+// no-op for a kernel launched the ordinary way.
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- thread-block clusters: hardware barrier and stores into a peer CTA's shared memory ----
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;

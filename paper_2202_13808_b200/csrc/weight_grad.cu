@@ -334,6 +334,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
+            ptx::grid_dependency_wait();   // the dense scratch is written by the kernel before this one
             int issued = 0;
             for (int i = 0; i < nkb && !*abort_flag; ++i) {
                 const int s = i % kStages;
@@ -593,14 +594,21 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     cfg.blockDim = dim3(kTcThreads);
     cfg.dynamicSmemBytes = kTcSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
+    cfg.attrs = attr;
     if (plan.cluster) {
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 1;
-        attr[0].val.clusterDim.y = (unsigned)plan.splits;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        attr[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
+        attr[cfg.numAttrs].val.clusterDim.x = 1;
+        attr[cfg.numAttrs].val.clusterDim.y = (unsigned)plan.splits;
+        attr[cfg.numAttrs].val.clusterDim.z = 1;
+        ++cfg.numAttrs;
+    }
+    if (plan.splits == 1 || plan.cluster) {
+        // the kernel right before this one in the stream is the decompression (no counter memset in
+        // between): this kernel may be set up while that one drains; it waits before reading the scratch
+        attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+        ++cfg.numAttrs;
     }
     if (cudaLaunchKernelEx(&cfg, wg_tc_kernel, map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n, plan.splits,
                            plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status,

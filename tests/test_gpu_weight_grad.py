@@ -25,6 +25,8 @@ SMALL = [
     di.small_linear(512, 256, 128, "bf16", 0.0),                       # gamma = 0: the dense gradient
     di.small_linear(512, 256, 128, "bf16", 1.0),                       # gamma = 1: zero gradient
     di.small_linear(8192, 256, 128, "bf16", 0.9),                      # one tile, deep split along tokens
+    di.small_linear(200, 2056, 1000, "bf16", 0.9),                     # 72 tiles x 2 splits: cluster of 2, ragged tiles
+    di.small_linear(512, 1792, 520, "bf16", 0.9),                      # 35 tiles x 4 splits: cluster of 4, ragged rows
 ]
 
 
@@ -90,8 +92,10 @@ def test_fused_weight_grad_full_size_and_unsupported(cuda_device):
         dropit.dropit_weight_grad(di.make_dy(small).to(cuda_device), c2, fused=True)
 
 
-def test_accumulate_adds_to_existing_gradient(cuda_device):
-    case = di.small_linear(640, 768, 384, "bf16", 0.9)
+@pytest.mark.parametrize("case", [di.small_linear(640, 768, 384, "bf16", 0.9),       # partial planes in global memory
+                                  di.small_linear(200, 2056, 1000, "bf16", 0.9)],    # cluster exchange
+                         ids=lambda c: c.name)
+def test_accumulate_adds_to_existing_gradient(cuda_device, case):
     bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
     base = torch.full_like(dw, 0.5)
     out = base.clone()
