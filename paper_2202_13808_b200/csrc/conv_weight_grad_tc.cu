@@ -82,6 +82,7 @@ struct ShiftDst {
 
 __global__ void __launch_bounds__(256)
 shift_copies_kernel(const uint4* __restrict__ in, ShiftDst dst, int64_t groups, int groups_per_row) {
+    ptx::launch_dependents();   // the GEMM behind this kernel may set itself up meanwhile
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += (int64_t)gridDim.x * blockDim.x) {
         const int gx = (int)(g % groups_per_row);
         const uint4 zero = make_uint4(0, 0, 0, 0);
@@ -112,6 +113,7 @@ __global__ void __launch_bounds__(256)
 conv_tc_reduce_kernel(const float* __restrict__ partial, int splits, int Cz, int Ca, int taps, float* __restrict__ dw,
                       int accumulate) {
     const int64_t plane = (int64_t)taps * Cz * Ca;
+    ptx::grid_dependency_wait();   // the partial tiles come from the kernel before this one
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < plane; i += (int64_t)gridDim.x * blockDim.x) {
         const int c = (int)(i % Ca);
         const int j = (int)((i / Ca) % Cz);
@@ -180,6 +182,7 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
 
     if (warp == 0) {
         if (lane == 0) {
+            ptx::grid_dependency_wait();   // the dense copies are written by the kernels before this one
             const uint32_t stage_bytes = (uint32_t)kAStageBytes + (uint32_t)ncols * 128u;
             int issued = 0;
             int xblk = kb_begin % p.nxb;
@@ -233,6 +236,7 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
             if (ok) ptx::umma_commit(&ctl->accum);
         }
     } else if (nkb > 0) {
+        ptx::launch_dependents();   // the reduction kernel may be brought up; it waits for this grid to finish
         bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
         ok = __all_sync(kFullMask, ok) && !*abort_flag;
         if (!ok) {
@@ -391,13 +395,33 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
     }
     float* partial = reinterpret_cast<float*>(ws + pl.partial_off);
     dim3 grid(pl.tiles, pl.p.splits);
-    conv_wg_tc_kernel<<<grid, kCThreads, kConvTcSmemBytes, stream>>>(maps, pl.p, partial, dev_status);
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kCThreads);
+    cfg.dynamicSmemBytes = kConvTcSmemBytes;
+    cfg.stream = stream;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, conv_wg_tc_kernel, maps, pl.p, partial, dev_status) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DROPIT_ERR_CUDA;
+    }
     st = check_launch();
     if (st != DROPIT_OK) return st;
     const int64_t count = (int64_t)R * S * Cz * Ca;
     int64_t blocks = (count + 255) / 256;
     if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
-    conv_tc_reduce_kernel<<<(unsigned)blocks, 256, 0, stream>>>(partial, pl.p.splits, Cz, Ca, R * S, dw, accumulate);
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    if (cudaLaunchKernelEx(&cfg, conv_tc_reduce_kernel, (const float*)partial, pl.p.splits, Cz, Ca, R * S, dw,
+                           accumulate) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DROPIT_ERR_CUDA;
+    }
     return check_launch();
 }
 
