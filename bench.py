@@ -283,7 +283,7 @@ def oracle_step(images: int, batch: int = 0) -> float:
     return secs
 
 
-def cpu_baseline_sample(images: int = 4):
+def cpu_baseline_sample(images: int = 48):
     import oracle
 
     oracle.build()
