@@ -18,6 +18,8 @@
 // When the band is wider than the per-warp histogram (small tensors, which are not sampled; key
 // distributions that are flat around T; a sample that missed) a general path is taken instead:
 // full CTA histogram in shared memory, global histogram by atomics, then one extra counting read.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace dropit {
@@ -336,6 +338,13 @@ __device__ __forceinline__ void ring_issue(uint32_t lane_slot, const uint4* x, i
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
+// The same for a block whose vectors are all whole: `src` = the lane's first vector of the block.
+__device__ __forceinline__ void ring_issue_full(uint32_t lane_slot, const uint4* src) {
+#pragma unroll
+    for (int j = 0; j < kVpl; ++j)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(lane_slot + j * 512), "l"(src + j * 32) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
 __device__ __forceinline__ void ring_read(uint32_t lane_slot, uint4 (&v)[kVpl]) {
 #pragma unroll
     for (int j = 0; j < kVpl; ++j)
@@ -400,6 +409,13 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     const int64_t blk0 = ((int64_t)blockIdx.x * kFusedWarps + warp) * blocks_per_warp;
     int64_t blk1 = blk0 + blocks_per_warp;
     if (blk1 > blocks_total) blk1 = blocks_total;
+    // blocks below this index consist of whole vectors only: they take the paths without bounds arithmetic
+    const int64_t blk_full_end = (nvec_full / kBlkVecs < blk1) ? nvec_full / kBlkVecs : blk1;
+    auto issue_block = [&](int64_t b, uint32_t dst) {
+        if (b < blk_full_end) ring_issue_full(dst, x + b * kBlkVecs + lane);
+        else if (b < blk1) ring_issue(dst, x, b, lane, nvec_full, n);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    };
     uint32_t barrier_target = 0;
 
     uint32_t lo = st->band_lo, hi = st->band_hi;
@@ -456,21 +472,21 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         if (narrow) {
             // stream the run through the ring, kRingDepth-1 blocks ahead
 #pragma unroll
-            for (int d = 0; d < kRingDepth - 1; ++d) {
-                if (blk0 + d < blk1) ring_issue(ring_lane + d * kRingSlotBytes, x, blk0 + d, lane, nvec_full, n);
-                else asm volatile("cp.async.commit_group;" ::: "memory");
-            }
+            for (int d = 0; d < kRingDepth - 1; ++d) issue_block(blk0 + d, ring_lane + d * kRingSlotBytes);
             int slot = 0, slot_ahead = kRingDepth - 1;
             for (int64_t blk = blk0; blk < blk1; ++blk) {
-                if (blk + kRingDepth - 1 < blk1)
-                    ring_issue(ring_lane + slot_ahead * kRingSlotBytes, x, blk + kRingDepth - 1, lane, nvec_full, n);
-                else asm volatile("cp.async.commit_group;" ::: "memory");
+                issue_block(blk + kRingDepth - 1, ring_lane + slot_ahead * kRingSlotBytes);
                 ring_wait();
                 uint4 va[kVpl];
                 ring_read(ring_lane + slot * kRingSlotBytes, va);
+                if (blk < blk_full_end) {
 #pragma unroll
-                for (int j = 0; j < kVpl; ++j)
-                    count_vec(va[j], valid_elems(blk * kBlkVecs + j * 32 + lane, nvec_full, n));
+                    for (int j = 0; j < kVpl; ++j) count_vec(va[j], 8);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kVpl; ++j)
+                        count_vec(va[j], valid_elems(blk * kBlkVecs + j * 32 + lane, nvec_full, n));
+                }
                 slot = (slot + 1 == kRingDepth) ? 0 : slot + 1;
                 slot_ahead = (slot_ahead + 1 == kRingDepth) ? 0 : slot_ahead + 1;
             }
@@ -718,25 +734,20 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     uint32_t pend = gpos & 7u, foreign = pend;       // staged-but-unwritten values; leading slots not ours
     uint32_t pend_i = gpos & 3u, foreign_i = pend_i;
 #pragma unroll
-    for (int d = 0; d < kRingDepth - 1; ++d) {
-        if (blk0 + d < blk1) ring_issue(ring_lane + d * kRingSlotBytes, x, blk0 + d, lane, nvec_full, n);
-        else asm volatile("cp.async.commit_group;" ::: "memory");
-    }
+    for (int d = 0; d < kRingDepth - 1; ++d) issue_block(blk0 + d, ring_lane + d * kRingSlotBytes);
     int slot = 0, slot_ahead = kRingDepth - 1;
-    for (int64_t blk = blk0; blk < blk1; ++blk) {
-        if (blk + kRingDepth - 1 < blk1)
-            ring_issue(ring_lane + slot_ahead * kRingSlotBytes, x, blk + kRingDepth - 1, lane, nvec_full, n);
-        else asm volatile("cp.async.commit_group;" ::: "memory");
+    // One block of the run.  FULL: every vector of the block is whole, so the bounds arithmetic folds away.
+    auto compact_block = [&](int64_t blk, auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
+        issue_block(blk + kRingDepth - 1, ring_lane + slot_ahead * kRingSlotBytes);
         ring_wait();
         uint4 cur[kVpl];
         ring_read(ring_lane + slot * kRingSlotBytes, cur);
         slot = (slot + 1 == kRingDepth) ? 0 : slot + 1;
         slot_ahead = (slot_ahead + 1 == kRingDepth) ? 0 : slot_ahead + 1;
-        int nvalid[kVpl];
         uint32_t gt8[kVpl], eq8[kVpl], cnt[kVpl];
 #pragma unroll
         for (int j = 0; j < kVpl; ++j) {
-            nvalid[j] = valid_elems(blk * kBlkVecs + j * 32 + lane, nvec_full, n);
             const uint32_t w[4] = {cur[j].x, cur[j].y, cur[j].z, cur[j].w};
             uint32_t a[4], eb[4], eany = 0;
 #pragma unroll
@@ -750,7 +761,10 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             uint32_t e8 = 0;
             if (eany & kHiBits) {
                 e8 = flags4(eb[0], eb[1]) | (flags4(eb[2], eb[3]) << 4);
-                e8 &= (1u << nvalid[j]) - 1u;   // zero padding past the end must not tie with T = 0
+                if constexpr (!FULL) {   // zero padding past the end must not tie with T = 0
+                    const int nvalid = valid_elems(blk * kBlkVecs + j * 32 + lane, nvec_full, n);
+                    e8 &= (1u << nvalid) - 1u;
+                }
             }
             gt8[j] = g8;
             eq8[j] = e8;
@@ -793,15 +807,20 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             }
             keep8[j] = gt8[j] | keep_eq;
             const uint32_t kept_before = gt_before + min(eq_before, q);
-            const int64_t vi = blk * kBlkVecs + j * 32 + lane;
-            if ((lane & 15) == 0 && vi * 8 < n) offsets[(vi * 8) / DROPIT_CHUNK] = kept_before;
+            if constexpr (FULL) {   // vector blk*64 + j*32 + lane opens chunk blk*4 + j*2 + lane/16 when lane % 16 == 0
+                if ((lane & 15) == 0) offsets[blk * (kBlkElems / DROPIT_CHUNK) + j * 2 + (lane >> 4)] = kept_before;
+            } else {
+                const int64_t vi = blk * kBlkVecs + j * 32 + lane;
+                if ((lane & 15) == 0 && vi * 8 < n) offsets[(vi * 8) / DROPIT_CHUNK] = kept_before;
+            }
             uint32_t pos = kept_before - blk_kept_base;
             const uint32_t w[4] = {cur[j].x, cur[j].y, cur[j].z, cur[j].w};
+            [[maybe_unused]] const int32_t first_idx = (int32_t)(blk * kBlkElems) + (j * 32 + lane) * 8;
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 if ((keep8[j] >> e) & 1u) {
                     s_vals[pend + pos] = (uint16_t)((w[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu);
-                    if constexpr (INDEX32) s_idx[pend_i + pos] = (int32_t)(vi * 8 + e);
+                    if constexpr (INDEX32) s_idx[pend_i + pos] = first_idx + e;
                     ++pos;
                 }
             }
@@ -824,7 +843,11 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                 if ((lane >> 3) == j) mine = got;
             }
             const int64_t w0 = blk * (kBlkElems / 32);
-            if (lane < 8 * kVpl && w0 + lane < nwords) mask[w0 + lane] = mine;
+            if constexpr (FULL) {
+                if (lane < 8 * kVpl) mask[w0 + lane] = mine;
+            } else {
+                if (lane < 8 * kVpl && w0 + lane < nwords) mask[w0 + lane] = mine;
+            }
         }
         const uint32_t kept = (run_gt + blk_gt + min(run_eq + blk_eq, q)) - blk_kept_base;
         run_gt += blk_gt;
@@ -833,6 +856,11 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         flush_pieces<uint16_t, 8>(s_vals, values + (gpos - pend), kept, pend, foreign, lane);
         if constexpr (INDEX32) flush_pieces<int32_t, 4>(s_idx, indices + (gpos - pend_i), kept, pend_i, foreign_i, lane);
         gpos += kept;
+    };
+    {
+        int64_t blk = blk0;
+        for (; blk < blk_full_end; ++blk) compact_block(blk, std::true_type{});
+        for (; blk < blk1; ++blk) compact_block(blk, std::false_type{});
     }
     // tails: own values still staged (less than one 16-byte piece); leading foreign slots are skipped
     if (lane >= (int)foreign && lane < (int)pend) values[(gpos - pend) + lane] = s_vals[lane];
