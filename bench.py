@@ -108,6 +108,11 @@ def algorithmic_bytes_compress(case) -> float:
     return 2 * n * 2 + n / 8 + k * 2 + 4 * ((n + 127) // 128)
 
 
+def compulsory_bytes_compress(case) -> float:
+    """One read of X plus the outputs: what any method has to move."""
+    return algorithmic_bytes_compress(case) - case.n * 2
+
+
 def dense_flops(case) -> float:
     return 2.0 * case.M * case.Ca * case.Cz
 
@@ -233,6 +238,8 @@ def run_ours(args, rank, world, device):
                               "achieved": comp_gbs[1], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                               "frac": comp_gbs[1] / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC["fused_compress_kernel_fc2"],
                               "peak_source": peaks["source"], "bytes_per_call": comp_bytes[1], "avg_ms": comp_ms[1],
+                              "compulsory_gbs": compulsory_bytes_compress(LAYERS[1]) / (comp_ms[1] * 1e-3) / 1e9,
+                              "dram_gbs": NCU_TRAFFIC["fused_compress_kernel_fc2"] / (comp_ms[1] * 1e-3) / 1e9,
                               "layer": LAYERS[1].name,
                               "other_layer": {"layer": LAYERS[0].name, "achieved": comp_gbs[0],
                                               "frac": comp_gbs[0] / peaks["hbm_gbs"], "avg_ms": comp_ms[0]}},
