@@ -109,6 +109,21 @@ bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same matrix seen as [cols / 64][rows][64]: one box {64, kBK, groups} brings `groups` adjacent 64-column
+// groups of kBK rows with a single copy, laid out group after group as the MN-major operand wants them.
+// Needs cols % 64 == 0 (a partial last group would read past the end of a row).
+static bool make_map_grouped_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int groups) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 2, 128};
+    cuuint32_t box[3] = {64, (cuuint32_t)kBK, (cuuint32_t)groups};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // ---------------------------------------------------------------------------------------------
 // tcgen05 kernel
 // ---------------------------------------------------------------------------------------------
@@ -289,7 +304,8 @@ __device__ __forceinline__ void cluster_finish_quarter(uint32_t tmem_base, const
 __global__ void __launch_bounds__(kTcThreads, 1)
 wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, int Ca, int Cz,
              int tiles_n, int splits, int kb_per_split, int kb_total, float* __restrict__ dw, int accumulate,
-             float* __restrict__ partial, uint32_t* counters, int32_t* dev_status, int cluster_mode) {
+             float* __restrict__ partial, uint32_t* counters, int32_t* dev_status, int cluster_mode,
+             int grouped_maps) {
     extern __shared__ uint8_t smem_raw[];
     // The dynamic window starts at the same offset in every CTA of the kernel, so this rounding gives
     // the same offsets in both CTAs of a cluster (the exchange below maps addresses between them).
@@ -346,10 +362,15 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
                 const int k0 = (kb_begin + i) * kBK;
                 uint8_t* a = sA + s * kAStageBytes;
                 uint8_t* b = sB + s * kBStageBytes;
+                if (grouped_maps) {   // one copy per operand
+                    ptx::tma_load_3d(a, &map_dy, 0, k0, j0 / 64, &ctl->full[s]);
+                    ptx::tma_load_3d(b, &map_x, 0, k0, c0 / 64, &ctl->full[s]);
+                } else {
 #pragma unroll
-                for (int g = 0; g < kBM / 64; ++g) ptx::tma_load_2d(a + g * (64 * kBK * 2), &map_dy, j0 + 64 * g, k0, &ctl->full[s]);
+                    for (int g = 0; g < kBM / 64; ++g) ptx::tma_load_2d(a + g * (64 * kBK * 2), &map_dy, j0 + 64 * g, k0, &ctl->full[s]);
 #pragma unroll
-                for (int g = 0; g < kBN / 64; ++g) ptx::tma_load_2d(b + g * (64 * kBK * 2), &map_x, c0 + 64 * g, k0, &ctl->full[s]);
+                    for (int g = 0; g < kBN / 64; ++g) ptx::tma_load_2d(b + g * (64 * kBK * 2), &map_x, c0 + 64 * g, k0, &ctl->full[s]);
+                }
                 issued = i + 1;
             }
             if (*abort_flag) {   // let the copies already in flight land before the CTA exits
@@ -576,7 +597,13 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     }
 
     CUtensorMap map_dy, map_x;
-    if (!make_map_2d_bf16(&map_dy, dy, M, Cz) || !make_map_2d_bf16(&map_x, dense, M, Ca)) return DROPIT_ERR_CUDA;
+    const bool grouped = (Ca % 64 == 0) && (Cz % 64 == 0);
+    if (grouped) {
+        if (!make_map_grouped_bf16(&map_dy, dy, M, Cz, kBM / 64) || !make_map_grouped_bf16(&map_x, dense, M, Ca, kBN / 64))
+            return DROPIT_ERR_CUDA;
+    } else if (!make_map_2d_bf16(&map_dy, dy, M, Cz) || !make_map_2d_bf16(&map_x, dense, M, Ca)) {
+        return DROPIT_ERR_CUDA;
+    }
     uint32_t* counters = reinterpret_cast<uint32_t*>(ws + plan.counters_off);
     float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
     if (plan.splits > 1 && !plan.cluster && cudaMemsetAsync(counters, 0, plan.counters_bytes, stream) != cudaSuccess)
@@ -612,7 +639,7 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     }
     if (cudaLaunchKernelEx(&cfg, wg_tc_kernel, map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n, plan.splits,
                            plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status,
-                           plan.cluster ? 1 : 0) != cudaSuccess) {
+                           plan.cluster ? 1 : 0, grouped ? 1 : 0) != cudaSuccess) {
         (void)cudaGetLastError();
         return DROPIT_ERR_CUDA;
     }
