@@ -23,7 +23,7 @@ constexpr int kMaxTapsX = 7;          // widest filter the tensor-core path take
 
 struct ConvMaps {
     CUtensorMap dy;
-    CUtensorMap x[kMaxTapsX];        // one per horizontal tap offset
+    CUtensorMap x;                   // all horizontally shifted copies: {W, H, C, B, tap}
 };
 
 struct ConvTcSmem {
@@ -61,6 +61,29 @@ bool make_map_nchw(CUtensorMap* map, const void* base, int B, int C, int H, int 
     cuuint32_t box[4] = {(cuuint32_t)xb, (cuuint32_t)yb, (cuuint32_t)rows, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+__device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            int c4, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(ptx::smem_u32(smem_dst)), "l"(map), "r"(ptx::smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+
+// The shifted copies lie `copy_stride` bytes apart: a fifth dimension over them lets one box {64, 1, rows, 1, taps}
+// bring the tiles of several horizontal taps, stacked tap after tap, with a single copy.
+bool make_map_taps(CUtensorMap* map, const void* base, int B, int C, int H, int W, int S, size_t copy_stride, int rows,
+                   int taps) {
+    EncodeTiledFn fn = conv_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[5] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)C, (cuuint64_t)B, (cuuint64_t)S};
+    cuuint64_t strides[4] = {(cuuint64_t)W * 2, (cuuint64_t)H * W * 2, (cuuint64_t)C * H * W * 2, (cuuint64_t)copy_stride};
+    cuuint32_t box[5] = {64, 1, (cuuint32_t)rows, 1, (cuuint32_t)taps};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -129,6 +152,7 @@ struct ConvTcParams {
     int Ca, Cz, R, S, pad;
     int xb, yb, nxb, nyb;        // k-block = xb x yb output positions (xb * yb = 64) of one image
     int bnc, nv, vgroups;        // B tile = nv horizontal taps x bnc input channels (nv * bnc <= 256)
+    int a_rows;                  // rows of dY the A copy brings (the rows of a 128-row tile that can exist)
     int tiles_c;
     int splits, kb_per_split, kb_total;
 };
@@ -168,7 +192,7 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
         ctl->abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&maps.dy);
-        for (int i = 0; i < nvt; ++i) ptx::prefetch_tensormap(&maps.x[v0 + i]);
+        ptx::prefetch_tensormap(&maps.x);
     }
     if (warp == 1) {
         ptx::tmem_alloc(&ctl->tmem_base, kBN);
@@ -183,7 +207,8 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
     if (warp == 0) {
         if (lane == 0) {
             ptx::grid_dependency_wait();   // the dense copies are written by the kernels before this one
-            const uint32_t stage_bytes = (uint32_t)kAStageBytes + (uint32_t)ncols * 128u;
+            // both boxes count in full, also where they reach outside the tensors (zero fill)
+            const uint32_t stage_bytes = (uint32_t)p.a_rows * 128u + (uint32_t)(p.nv * p.bnc) * 128u;
             int issued = 0;
             int xblk = kb_begin % p.nxb;
             int yblk = (kb_begin / p.nxb) % p.nyb;
@@ -197,9 +222,7 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
                 ptx::mbar_arrive_expect_tx(&ctl->full[s], stage_bytes);
                 const int x0 = xblk * p.xb, y0 = yblk * p.yb;
                 tma_load_4d(sA + s * kAStageBytes, &maps.dy, x0, y0, j0, n, &ctl->full[s]);
-                uint8_t* b = sB + s * kBStageBytes;
-                for (int i2 = 0; i2 < nvt; ++i2)
-                    tma_load_4d(b + (size_t)i2 * p.bnc * 128, &maps.x[v0 + i2], x0, y0 + u - p.pad, c0, n, &ctl->full[s]);
+                tma_load_5d(sB + s * kBStageBytes, &maps.x, x0, y0 + u - p.pad, c0, n, v0, &ctl->full[s]);
                 issued = i + 1;
                 if (++xblk == p.nxb) {
                     xblk = 0;
@@ -328,6 +351,7 @@ ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, 
     if (p.nv < 1) p.nv = 1;
     p.vgroups = (S + p.nv - 1) / p.nv;
     p.tiles_c = (Ca + p.bnc - 1) / p.bnc;
+    p.a_rows = Cz >= kBM ? kBM : (Cz + 7) / 8 * 8;   // tile rows past these hold stale bytes and feed unused D rows
     const int64_t tiles = (int64_t)((Cz + kBM - 1) / kBM) * p.tiles_c * R * p.vgroups;
     if (tiles > (1ll << 30)) return pl;
     pl.tiles = (int)tiles;
@@ -381,11 +405,8 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
         if (st != DROPIT_OK) return st;
     }
     ConvMaps maps;
-    if (!make_map_nchw(&maps.dy, dy, B, Cz, pl.Ho, pl.Wo, pl.p.xb, pl.p.yb, kBM)) return DROPIT_ERR_CUDA;
-    for (int v = 0; v < S; ++v)
-        if (!make_map_nchw(&maps.x[v], ws + pl.dense_stride * v, B, Ca, pl.H, pl.W, pl.p.xb, pl.p.yb, pl.p.bnc))
-            return DROPIT_ERR_CUDA;
-    for (int v = S; v < kMaxTapsX; ++v) maps.x[v] = maps.x[0];   // never read; keeps the parameter defined
+    if (!make_map_nchw(&maps.dy, dy, B, Cz, pl.Ho, pl.Wo, pl.p.xb, pl.p.yb, pl.p.a_rows)) return DROPIT_ERR_CUDA;
+    if (!make_map_taps(&maps.x, ws, B, Ca, pl.H, pl.W, S, pl.dense_stride, pl.p.bnc, pl.p.nv)) return DROPIT_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(conv_wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
