@@ -21,6 +21,7 @@
 #include <type_traits>
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace dropit {
 
@@ -147,6 +148,7 @@ sample_band_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long k,
     unsigned long long t_begin;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_begin));
 #endif
+    ptx::grid_dependency_wait();   // launched programmatically: x may come from the kernel before this one
     const int64_t nvec = n / 8;
     const bool sampled = n >= kSampleMinElems;
     uint4 sv[kSampleVecs / kSampleThreads];
@@ -726,6 +728,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     phase_stamp(st, 3);
 
     // ---------------- phase 3: ordered compaction, one warp per run of blocks ----------------
+    ptx::launch_dependents();   // a programmatically launched kernel behind this one may be brought up
     const int64_t nwords = (n + 31) / 32;
     uint16_t* s_vals = s_vals_all + (size_t)warp * kStageVals;
     int32_t* s_idx = s_idx_all + (size_t)warp * kStageIdx;
@@ -891,8 +894,23 @@ dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool inde
             return DROPIT_ERR_CUDA;
         attr_set = true;
     }
-    sample_band_kernel<<<1, kSampleThreads, smem_hist, stream>>>(reinterpret_cast<const uint4*>(x), n,
-                                                               (unsigned long long)k, ws, plan.zero_bytes);
+    {
+        cudaLaunchAttribute pdl[1];
+        pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        pdl[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1);
+        cfg.blockDim = dim3(kSampleThreads);
+        cfg.dynamicSmemBytes = smem_hist;
+        cfg.stream = stream;
+        cfg.attrs = pdl;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, sample_band_kernel, reinterpret_cast<const uint4*>(x), n, (unsigned long long)k, ws,
+                               plan.zero_bytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return DROPIT_ERR_CUDA;
+        }
+    }
     dropit_status s = check_launch();
     if (s != DROPIT_OK) return s;
 

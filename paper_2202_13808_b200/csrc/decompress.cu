@@ -22,7 +22,8 @@ decompress_bitmask_kernel(const typename Tr::elem_t* __restrict__ values, const 
     constexpr int kPitch = 32 + G;                   // image row = one mask word; one spare vector spreads the banks
     constexpr int kVecPerRow = 32 / G;
     __shared__ __align__(16) elem_t image[kDecompWarps][32 * kPitch];
-    ptx::launch_dependents();   // a weight-gradient kernel behind this one may set itself up meanwhile
+    ptx::grid_dependency_wait();   // launched programmatically: the cache may come from the kernel before this one
+    ptx::launch_dependents();      // a weight-gradient kernel behind this one may set itself up meanwhile
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     elem_t* img = image[warp];
     const int64_t nwords = (n + 31) / 32;
@@ -72,6 +73,7 @@ template <typename Tr>
 __global__ void __launch_bounds__(256)
 scatter_index32_kernel(const typename Tr::elem_t* __restrict__ values, const int32_t* __restrict__ idx, int64_t k,
                        int64_t n, typename Tr::elem_t* __restrict__ out) {
+    ptx::grid_dependency_wait();
     ptx::launch_dependents();
     for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < k; r += (int64_t)gridDim.x * blockDim.x) {
         const int64_t i = idx[r];
@@ -88,9 +90,22 @@ static dropit_status run_decompress(const void* values, const void* meta, const 
         const int64_t ntiles = (n + 1023) / 1024;       // one warp step each
         int64_t blocks = (ntiles + kDecompWarps - 1) / kDecompWarps;
         if (blocks > cap * 4) blocks = cap * 4;
-        decompress_bitmask_kernel<Tr><<<(unsigned)blocks, 32 * kDecompWarps, 0, stream>>>(
-            reinterpret_cast<const elem_t*>(values), reinterpret_cast<const uint32_t*>(meta), offsets, n,
-            reinterpret_cast<elem_t*>(out));
+        // programmatic launch: the kernel may be brought up while the one before it drains; it waits at its top
+        cudaLaunchAttribute pdl[1];
+        pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        pdl[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks);
+        cfg.blockDim = dim3(32 * kDecompWarps);
+        cfg.stream = stream;
+        cfg.attrs = pdl;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, decompress_bitmask_kernel<Tr>, reinterpret_cast<const elem_t*>(values),
+                               reinterpret_cast<const uint32_t*>(meta), offsets, n, reinterpret_cast<elem_t*>(out)) !=
+            cudaSuccess) {
+            (void)cudaGetLastError();
+            return DROPIT_ERR_CUDA;
+        }
         return check_launch();
     }
     if (cudaMemsetAsync(out, 0, (size_t)n * Tr::kElemBytes, stream) != cudaSuccess) return DROPIT_ERR_CUDA;

@@ -406,6 +406,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         }
     } else {
         // ---------------- epilogue: TMEM -> global ----------------
+        ptx::launch_dependents();   // a programmatically launched kernel behind this one may be brought up
         bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
         ok = __all_sync(kFullMask, ok) && !*abort_flag;
         if (!ok) *abort_flag = 1;
