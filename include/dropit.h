@@ -178,8 +178,8 @@ dropit_status dropit_weight_grad(const void* dy, const void* values, const void*
  * R(a-hat) tiles (Sec. 3.2) are built there, right in front of the tensor cores.  Needs
  * dtype = DROPIT_BF16, format = DROPIT_FMT_BITMASK, Ca a multiple of 128 and Cz a multiple of 8;
  * anything else returns DROPIT_ERR_UNSUPPORTED.  Same arguments and workspace size as
- * dropit_weight_grad.  On B200 it is currently the slower of the two variants; dropit_weight_grad
- * chooses between them.
+ * dropit_weight_grad, of which it uses less (no dense scratch is touched).  On B200 it is the
+ * slower of the two variants; dropit_weight_grad never takes it on its own.
  */
 dropit_status dropit_weight_grad_fused(const void* dy, const void* values, const void* meta, const uint32_t* offsets,
                                        int64_t M, int64_t Ca, int64_t Cz, int64_t k, dropit_dtype dtype,
@@ -199,6 +199,10 @@ dropit_status dropit_conv_weight_grad_workspace(int B, int Ca, int H, int W, int
  *   dy [device, B x Cz x Ho x Wo, dtype] with Ho = (H + 2 pad - R)/stride + 1,
  *   Wo likewise; values/meta/offsets [device] = cache of a [B x Ca x H x W];
  *   dw [device, Cz x Ca x R x S, float], overwritten or accumulated into.
+ * bf16 with stride 1, S <= 7 and Wo <= W runs on the tensor cores (one implicit GEMM per
+ * filter tap over (n, y, x), fp32 accumulation, fixed summation order); other shapes and
+ * fp32 inputs use an fp32 FMA kernel.  A bounded device wait that expires is reported
+ * through dev_status as DROPIT_ERR_TIMEOUT.
  */
 dropit_status dropit_conv_weight_grad(const void* dy, const void* values, const void* meta, const uint32_t* offsets,
                                       int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad,

@@ -131,6 +131,27 @@ shift_copies_kernel(const uint4* __restrict__ in, ShiftDst dst, int64_t groups, 
     }
 }
 
+// Rows that are not a multiple of 8 pixels cannot be TMA rows (strides are multiples of 16 bytes): this
+// kernel rewrites a [rows, W] tensor with row pitch Wp (a multiple of 8, zero padded), once per destination,
+// shifted like shift_copies_kernel.  dst.out is indexed by shift + kMaxTapsX - 1 as there, shift 0 included.
+__global__ void __launch_bounds__(256)
+pad_shift_rows_kernel(const uint16_t* __restrict__ in, ShiftDst dst, int64_t rows, int W, int Wp) {
+    ptx::launch_dependents();
+    const int64_t total = rows * Wp;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / Wp;
+        const int x = (int)(i - row * Wp);
+        const uint16_t* src = in + row * W;
+#pragma unroll
+        for (int sh = -(kMaxTapsX - 1); sh <= kMaxTapsX - 1; ++sh) {
+            uint16_t* out = reinterpret_cast<uint16_t*>(dst.out[sh + kMaxTapsX - 1]);
+            if (out == nullptr) continue;
+            const int xs = x + sh;
+            out[i] = (x < W && xs >= 0 && xs < W) ? src[xs] : (uint16_t)0;
+        }
+    }
+}
+
 // dw[j,c,u,v] (=|+=) sum over splits of partial[split][tap][j][c]
 __global__ void __launch_bounds__(256)
 conv_tc_reduce_kernel(const float* __restrict__ partial, int splits, int Cz, int Ca, int taps, float* __restrict__ dw,
@@ -324,7 +345,9 @@ struct ConvTcPlan {
     int H, W, Ho, Wo;          // geometry the kernel sees (a 1x1 filter flattens each plane into one row)
     int tiles;
     ConvTcParams p;
-    size_t dense_stride, partial_off, total_bytes;
+    bool padded;               // rows are not multiples of 8 pixels: the GEMM reads zero-padded copies of X and dY
+    int Wp, Wop;               // row pitch of the X copies / of the dY the GEMM reads
+    size_t dense_stride, tmp_off, dy_off, partial_off, total_bytes;
 };
 
 ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad, dropit_dtype dtype) {
@@ -334,7 +357,10 @@ ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, 
     if (R == 1 && S == 1 && pad == 0) {   // plain GEMM over the flattened plane
         W = H * W; H = 1; Wo = W; Ho = 1;
     }
-    if (Wo > W || (W & 7) || (Wo & 7)) return pl;   // TMA strides are multiples of 16 bytes
+    if (Wo > W) return pl;
+    pl.padded = (W & 7) || (Wo & 7);               // TMA strides are multiples of 16 bytes
+    pl.Wp = (W + 7) / 8 * 8;
+    pl.Wop = (Wo + 7) / 8 * 8;
     ConvTcParams& p = pl.p;
     p.Ca = Ca; p.Cz = Cz; p.R = R; p.S = S; p.pad = pad;
     // One k-block = 64 consecutive pixels of one image row, so a tile row is exactly one 128-byte
@@ -362,8 +388,10 @@ ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, 
     p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
     if (p.splits > 65535) return pl;
     pl.H = H; pl.W = W; pl.Ho = Ho; pl.Wo = Wo;
-    pl.dense_stride = align_up((size_t)B * Ca * H * W * 2, 256);
-    pl.partial_off = pl.dense_stride * S;
+    pl.dense_stride = align_up((size_t)B * Ca * H * pl.Wp * 2, 256);
+    pl.tmp_off = pl.dense_stride * S;
+    pl.dy_off = pl.tmp_off + (pl.padded ? align_up((size_t)B * Ca * H * W * 2, 256) : 0);
+    pl.partial_off = pl.dy_off + (pl.padded ? align_up((size_t)B * Cz * Ho * pl.Wop * 2, 256) : 0);
     pl.total_bytes = pl.partial_off + align_up((size_t)p.splits * R * S * Cz * Ca * 4, 256);
     pl.ok = true;
     return pl;
@@ -388,25 +416,54 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
     if (workspace_bytes < pl.total_bytes) return DROPIT_ERR_WORKSPACE;
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
     const int64_t n = (int64_t)B * Ca * H * W;
-    // the unshifted copy lives in slot `pad`, so slot v always holds the rows shifted by v - pad
-    void* dense0 = ws + pl.dense_stride * pad;
-    dropit_status st = decompress_dispatch(values, meta, offsets, n, k, DROPIT_BF16, format, dense0, stream);
-    if (st != DROPIT_OK) return st;
-    if (S > 1) {
+    // slot v of the scratch holds the rows shifted by v - pad
+    const void* dy_gemm = dy;
+    if (!pl.padded) {
+        void* dense0 = ws + pl.dense_stride * pad;   // the unshifted copy is the decompressed tensor itself
+        dropit_status st0 = decompress_dispatch(values, meta, offsets, n, k, DROPIT_BF16, format, dense0, stream);
+        if (st0 != DROPIT_OK) return st0;
+        if (S > 1) {
+            ShiftDst dst{};
+            for (int v = 0; v < S; ++v)
+                if (v != pad) dst.out[v - pad + kMaxTapsX - 1] = reinterpret_cast<uint4*>(ws + pl.dense_stride * v);
+            const int64_t groups = n / 8;
+            int64_t blocks = (groups + 255) / 256;
+            if (blocks > (int64_t)sm_count() * 16) blocks = (int64_t)sm_count() * 16;
+            shift_copies_kernel<<<(unsigned)blocks, 256, 0, stream>>>(reinterpret_cast<const uint4*>(dense0), dst, groups,
+                                                                     pl.W / 8);
+            st0 = check_launch();
+            if (st0 != DROPIT_OK) return st0;
+        }
+    } else {
+        uint16_t* tmp = reinterpret_cast<uint16_t*>(ws + pl.tmp_off);
+        dropit_status st0 = decompress_dispatch(values, meta, offsets, n, k, DROPIT_BF16, format, tmp, stream);
+        if (st0 != DROPIT_OK) return st0;
+        const int cap = sm_count() * 16;
+        {   // dY with padded rows
+            ShiftDst dst{};
+            dst.out[kMaxTapsX - 1] = reinterpret_cast<uint4*>(ws + pl.dy_off);
+            const int64_t rows = (int64_t)B * Cz * pl.Ho;
+            int64_t blocks = (rows * pl.Wop + 255) / 256;
+            if (blocks > cap) blocks = cap;
+            pad_shift_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(reinterpret_cast<const uint16_t*>(dy), dst, rows,
+                                                                       pl.Wo, pl.Wop);
+            st0 = check_launch();
+            if (st0 != DROPIT_OK) return st0;
+            dy_gemm = ws + pl.dy_off;
+        }
         ShiftDst dst{};
-        for (int v = 0; v < S; ++v)
-            if (v != pad) dst.out[v - pad + kMaxTapsX - 1] = reinterpret_cast<uint4*>(ws + pl.dense_stride * v);
-        const int64_t groups = n / 8;
-        int64_t blocks = (groups + 255) / 256;
-        if (blocks > (int64_t)sm_count() * 16) blocks = (int64_t)sm_count() * 16;
-        shift_copies_kernel<<<(unsigned)blocks, 256, 0, stream>>>(reinterpret_cast<const uint4*>(dense0), dst, groups,
-                                                                 pl.W / 8);
-        st = check_launch();
-        if (st != DROPIT_OK) return st;
+        for (int v = 0; v < S; ++v) dst.out[v - pad + kMaxTapsX - 1] = reinterpret_cast<uint4*>(ws + pl.dense_stride * v);
+        const int64_t rows = (int64_t)B * Ca * pl.H;
+        int64_t blocks = (rows * pl.Wp + 255) / 256;
+        if (blocks > cap) blocks = cap;
+        pad_shift_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(tmp, dst, rows, pl.W, pl.Wp);
+        st0 = check_launch();
+        if (st0 != DROPIT_OK) return st0;
     }
+    dropit_status st = DROPIT_OK;
     ConvMaps maps;
-    if (!make_map_nchw(&maps.dy, dy, B, Cz, pl.Ho, pl.Wo, pl.p.xb, pl.p.yb, pl.p.a_rows)) return DROPIT_ERR_CUDA;
-    if (!make_map_taps(&maps.x, ws, B, Ca, pl.H, pl.W, S, pl.dense_stride, pl.p.bnc, pl.p.nv)) return DROPIT_ERR_CUDA;
+    if (!make_map_nchw(&maps.dy, dy_gemm, B, Cz, pl.Ho, pl.Wop, pl.p.xb, pl.p.yb, pl.p.a_rows)) return DROPIT_ERR_CUDA;
+    if (!make_map_taps(&maps.x, ws, B, Ca, pl.H, pl.Wp, S, pl.dense_stride, pl.p.bnc, pl.p.nv)) return DROPIT_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(conv_wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

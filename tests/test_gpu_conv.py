@@ -32,6 +32,9 @@ SMALL = [
     di.small_conv(1, 16, 4, 72, 16, 3, 3, 1, 1, "bf16", 0.8),        # rows wider than one k-block
     di.small_conv(2, 3, 16, 16, 8, 7, 7, 1, 3, "bf16", 0.5),         # 7x7 on 3 channels
     di.small_conv(150, 8, 8, 8, 8, 3, 3, 1, 1, "bf16", 0.8),         # more k-blocks than splits, uneven
+    di.small_conv(4, 256, 14, 14, 256, 3, 3, 1, 1, "bf16", 0.8),     # ResNet stage-3 shape: rows padded to 16 pixels
+    di.small_conv(4, 512, 7, 7, 128, 1, 1, 1, 0, "bf16", 0.8),       # 7x7 planes flattened to 49 -> 56 pixels
+    di.small_conv(2, 24, 11, 13, 24, 5, 3, 1, 1, "bf16", 0.5),       # Ho != H, Wo = W, odd sizes, non-square filter
     di.small_conv(4, 64, 56, 56, 64, 3, 3, 1, 1, "bf16", 0.8),       # the ResNet stage-1 3x3 shape, 4 images
     di.small_conv(4, 256, 56, 56, 64, 1, 1, 1, 0, "bf16", 0.8),      # the ResNet stage-1 1x1 shape, 4 images
 ]
