@@ -199,7 +199,7 @@ dropit_status dropit_conv_weight_grad_workspace(int B, int Ca, int H, int W, int
  *   dy [device, B x Cz x Ho x Wo, dtype] with Ho = (H + 2 pad - R)/stride + 1,
  *   Wo likewise; values/meta/offsets [device] = cache of a [B x Ca x H x W];
  *   dw [device, Cz x Ca x R x S, float], overwritten or accumulated into.
- * bf16 with stride 1, S <= 7 and Wo <= W runs on the tensor cores (one implicit GEMM per
+ * bf16 with S <= 7 (and Wo <= W when stride is 1) runs on the tensor cores (one implicit GEMM per
  * filter tap over (n, y, x), fp32 accumulation, fixed summation order); other shapes and
  * fp32 inputs use an fp32 FMA kernel.  A bounded device wait that expires is reported
  * through dev_status as DROPIT_ERR_TIMEOUT.

@@ -152,6 +152,31 @@ pad_shift_rows_kernel(const uint16_t* __restrict__ in, ShiftDst dst, int64_t row
     }
 }
 
+// Strided convolutions: one copy of the input per filter tap, sampled at the output positions,
+//   out[t = u*S + v][n,c,y,x] = in[n,c, y*stride + u - pad, x*stride + v - pad]   (0 outside the image),
+// with output geometry [Ho, Wp] (row pitch a multiple of 8 pixels, zero padded).  After this every tap is a plain
+// GEMM of dY against its own copy.
+__global__ void __launch_bounds__(256)
+gather_taps_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, size_t copy_elems, int64_t planes,
+                   int H, int W, int Ho, int Wo, int Wp, int R, int S, int stride, int pad) {
+    ptx::launch_dependents();
+    const int64_t total = planes * Ho * Wp;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int x = (int)(i % Wp);
+        const int y = (int)((i / Wp) % Ho);
+        const int64_t plane = i / ((int64_t)Wp * Ho);
+        const uint16_t* src = in + plane * H * W;
+        for (int u = 0; u < R; ++u) {
+            const int yi = y * stride + u - pad;
+            for (int v = 0; v < S; ++v) {
+                const int xi = x * stride + v - pad;
+                const bool ok = x < Wo && yi >= 0 && yi < H && xi >= 0 && xi < W;
+                out[(size_t)(u * S + v) * copy_elems + i] = ok ? src[(int64_t)yi * W + xi] : (uint16_t)0;
+            }
+        }
+    }
+}
+
 // dw[j,c,u,v] (=|+=) sum over splits of partial[split][tap][j][c]
 __global__ void __launch_bounds__(256)
 conv_tc_reduce_kernel(const float* __restrict__ partial, int splits, int Cz, int Ca, int taps, float* __restrict__ dw,
@@ -174,6 +199,7 @@ struct ConvTcParams {
     int xb, yb, nxb, nyb;        // k-block = xb x yb output positions (xb * yb = 64) of one image
     int bnc, nv, vgroups;        // B tile = nv horizontal taps x bnc input channels (nv * bnc <= 256)
     int a_rows;                  // rows of dY the A copy brings (the rows of a 128-row tile that can exist)
+    int gathered;                // strided filter: the scratch holds one pre-sampled copy per tap (u*S + v)
     int tiles_c;
     int splits, kb_per_split, kb_total;
 };
@@ -243,7 +269,8 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
                 ptx::mbar_arrive_expect_tx(&ctl->full[s], stage_bytes);
                 const int x0 = xblk * p.xb, y0 = yblk * p.yb;
                 tma_load_4d(sA + s * kAStageBytes, &maps.dy, x0, y0, j0, n, &ctl->full[s]);
-                tma_load_5d(sB + s * kBStageBytes, &maps.x, x0, y0 + u - p.pad, c0, n, v0, &ctl->full[s]);
+                if (p.gathered) tma_load_5d(sB + s * kBStageBytes, &maps.x, x0, y0, c0, n, u * p.S + v0, &ctl->full[s]);
+                else tma_load_5d(sB + s * kBStageBytes, &maps.x, x0, y0 + u - p.pad, c0, n, v0, &ctl->full[s]);
                 issued = i + 1;
                 if (++xblk == p.nxb) {
                     xblk = 0;
@@ -345,24 +372,32 @@ struct ConvTcPlan {
     int H, W, Ho, Wo;          // geometry the kernel sees (a 1x1 filter flattens each plane into one row)
     int tiles;
     ConvTcParams p;
-    bool padded;               // rows are not multiples of 8 pixels: the GEMM reads zero-padded copies of X and dY
+    bool padded;               // the GEMM reads rewritten copies of X (rows not multiples of 8 pixels, or a strided filter)
+    bool pad_dy;               // ... and a zero-padded copy of dY
+    int copies;                // copies of X in the scratch: S (one per horizontal tap) or R*S (strided filter)
+    int Hx;                    // rows per plane of the X copies
     int Wp, Wop;               // row pitch of the X copies / of the dY the GEMM reads
     size_t dense_stride, tmp_off, dy_off, partial_off, total_bytes;
 };
 
 ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, int stride, int pad, dropit_dtype dtype) {
     ConvTcPlan pl{};
-    if (dtype != DROPIT_BF16 || stride != 1 || S > kMaxTapsX || pad > kMaxTapsX - 1 || B < 1) return pl;
-    int Ho = H + 2 * pad - R + 1, Wo = W + 2 * pad - S + 1;
-    if (R == 1 && S == 1 && pad == 0) {   // plain GEMM over the flattened plane
+    if (dtype != DROPIT_BF16 || S > kMaxTapsX || pad > kMaxTapsX - 1 || B < 1) return pl;
+    int Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
+    const bool gathered = stride != 1;
+    if (!gathered && R == 1 && S == 1 && pad == 0) {   // plain GEMM over the flattened plane
         W = H * W; H = 1; Wo = W; Ho = 1;
     }
-    if (Wo > W) return pl;
-    pl.padded = (W & 7) || (Wo & 7);               // TMA strides are multiples of 16 bytes
-    pl.Wp = (W + 7) / 8 * 8;
+    if (!gathered && Wo > W) return pl;
+    pl.padded = gathered || (W & 7) || (Wo & 7);   // TMA strides are multiples of 16 bytes
+    pl.pad_dy = (Wo & 7) != 0;
+    pl.copies = gathered ? R * S : S;
+    pl.Hx = gathered ? Ho : H;
+    pl.Wp = ((gathered ? Wo : W) + 7) / 8 * 8;
     pl.Wop = (Wo + 7) / 8 * 8;
     ConvTcParams& p = pl.p;
     p.Ca = Ca; p.Cz = Cz; p.R = R; p.S = S; p.pad = pad;
+    p.gathered = gathered ? 1 : 0;
     // One k-block = 64 consecutive pixels of one image row, so a tile row is exactly one 128-byte
     // swizzle row.  (Boxes with a narrower inner extent and several image rows are not used: their
     // shared-memory footprint under the 128-byte swizzle is not the dense one.)
@@ -388,10 +423,10 @@ ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, 
     p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
     if (p.splits > 65535) return pl;
     pl.H = H; pl.W = W; pl.Ho = Ho; pl.Wo = Wo;
-    pl.dense_stride = align_up((size_t)B * Ca * H * pl.Wp * 2, 256);
-    pl.tmp_off = pl.dense_stride * S;
+    pl.dense_stride = align_up((size_t)B * Ca * pl.Hx * pl.Wp * 2, 256);
+    pl.tmp_off = pl.dense_stride * pl.copies;
     pl.dy_off = pl.tmp_off + (pl.padded ? align_up((size_t)B * Ca * H * W * 2, 256) : 0);
-    pl.partial_off = pl.dy_off + (pl.padded ? align_up((size_t)B * Cz * Ho * pl.Wop * 2, 256) : 0);
+    pl.partial_off = pl.dy_off + (pl.pad_dy ? align_up((size_t)B * Cz * Ho * pl.Wop * 2, 256) : 0);
     pl.total_bytes = pl.partial_off + align_up((size_t)p.splits * R * S * Cz * Ca * 4, 256);
     pl.ok = true;
     return pl;
@@ -439,7 +474,7 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
         dropit_status st0 = decompress_dispatch(values, meta, offsets, n, k, DROPIT_BF16, format, tmp, stream);
         if (st0 != DROPIT_OK) return st0;
         const int cap = sm_count() * 16;
-        {   // dY with padded rows
+        if (pl.pad_dy) {   // dY with padded rows
             ShiftDst dst{};
             dst.out[kMaxTapsX - 1] = reinterpret_cast<uint4*>(ws + pl.dy_off);
             const int64_t rows = (int64_t)B * Cz * pl.Ho;
@@ -451,19 +486,30 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
             if (st0 != DROPIT_OK) return st0;
             dy_gemm = ws + pl.dy_off;
         }
-        ShiftDst dst{};
-        for (int v = 0; v < S; ++v) dst.out[v - pad + kMaxTapsX - 1] = reinterpret_cast<uint4*>(ws + pl.dense_stride * v);
-        const int64_t rows = (int64_t)B * Ca * pl.H;
-        int64_t blocks = (rows * pl.Wp + 255) / 256;
-        if (blocks > cap) blocks = cap;
-        pad_shift_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(tmp, dst, rows, pl.W, pl.Wp);
+        if (pl.p.gathered) {
+            const int64_t planes = (int64_t)B * Ca;
+            int64_t blocks = (planes * pl.Ho * pl.Wp + 255) / 256;
+            if (blocks > cap) blocks = cap;
+            gather_taps_kernel<<<(unsigned)blocks, 256, 0, stream>>>(tmp, reinterpret_cast<uint16_t*>(ws),
+                                                                    pl.dense_stride / 2, planes, H, W, pl.Ho, pl.Wo,
+                                                                    pl.Wp, R, S, stride, pad);
+        } else {
+            ShiftDst dst{};
+            for (int v = 0; v < S; ++v)
+                dst.out[v - pad + kMaxTapsX - 1] = reinterpret_cast<uint4*>(ws + pl.dense_stride * v);
+            const int64_t rows = (int64_t)B * Ca * pl.H;
+            int64_t blocks = (rows * pl.Wp + 255) / 256;
+            if (blocks > cap) blocks = cap;
+            pad_shift_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(tmp, dst, rows, pl.W, pl.Wp);
+        }
         st0 = check_launch();
         if (st0 != DROPIT_OK) return st0;
     }
     dropit_status st = DROPIT_OK;
     ConvMaps maps;
     if (!make_map_nchw(&maps.dy, dy_gemm, B, Cz, pl.Ho, pl.Wop, pl.p.xb, pl.p.yb, pl.p.a_rows)) return DROPIT_ERR_CUDA;
-    if (!make_map_taps(&maps.x, ws, B, Ca, pl.H, pl.Wp, S, pl.dense_stride, pl.p.bnc, pl.p.nv)) return DROPIT_ERR_CUDA;
+    if (!make_map_taps(&maps.x, ws, B, Ca, pl.Hx, pl.Wp, pl.copies, pl.dense_stride, pl.p.bnc, pl.p.nv))
+        return DROPIT_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(conv_wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -35,6 +35,10 @@ SMALL = [
     di.small_conv(4, 256, 14, 14, 256, 3, 3, 1, 1, "bf16", 0.8),     # ResNet stage-3 shape: rows padded to 16 pixels
     di.small_conv(4, 512, 7, 7, 128, 1, 1, 1, 0, "bf16", 0.8),       # 7x7 planes flattened to 49 -> 56 pixels
     di.small_conv(2, 24, 11, 13, 24, 5, 3, 1, 1, "bf16", 0.5),       # Ho != H, Wo = W, odd sizes, non-square filter
+    di.small_conv(2, 16, 16, 16, 24, 3, 3, 2, 1, "bf16", 0.8),       # stride 2: one pre-sampled copy per tap
+    di.small_conv(2, 8, 15, 15, 8, 1, 1, 2, 0, "bf16", 0.8),         # 1x1 stride 2 (shortcut), odd image
+    di.small_conv(1, 3, 32, 32, 16, 7, 7, 2, 3, "bf16", 0.5),        # 7x7 stride 2 pad 3 on 3 channels (stem)
+    di.small_conv(2, 130, 28, 28, 140, 3, 3, 2, 1, "bf16", 0.8),     # stride 2, two row tiles, ragged channels
     di.small_conv(4, 64, 56, 56, 64, 3, 3, 1, 1, "bf16", 0.8),       # the ResNet stage-1 3x3 shape, 4 images
     di.small_conv(4, 256, 56, 56, 64, 1, 1, 1, 0, "bf16", 0.8),      # the ResNet stage-1 1x1 shape, 4 images
 ]
