@@ -138,8 +138,8 @@ struct TcSmem {
 constexpr int kEpiRowFloats = 36;                          // staging row pitch: 32 columns + 4 (bank spread, 16-byte rows)
 constexpr int kEpiWarpFloats = 32 * kEpiRowFloats;         // one warp's 32 x 32 chunk
 constexpr int kEpiSpinLimit = 1 << 20;
-constexpr int kXchgRowFloats = kBN + 4;                    // exchange row pitch: lanes of a warp (rows) hit distinct banks
-constexpr int kXchgMaxBytes = 3 * 32 * kXchgRowFloats * 4; // 4 splits: three peers send 32 rows each (2 splits: one sends 64)
+// cluster exchange, receive area: (splits - 1) slots x 128 rows x (256 / splits + 4) floats; largest for 4 splits
+constexpr int kXchgMaxBytes = 3 * kBM * (kBN / 4 + 4) * 4;
 constexpr size_t kTcSmemBytes = 1024 + (size_t)kStages * (kAStageBytes + kBStageBytes) + sizeof(TcSmem);
 
 // Epilogue of one 128 x 256 accumulator tile, run by the four warps that own the TMEM lane quarters.
@@ -225,40 +225,44 @@ __device__ __forceinline__ void epilogue_tile_staged(uint32_t tmem_base, float* 
 }
 
 // Split reduction inside a thread-block cluster (2 or 4 splits of one tile are the CTAs of one cluster).
-// The tile's four 32-row quarters are shared out among the CTAs; every CTA sends the quarters it does
-// not own from TMEM into the owner's shared memory, the owner adds the terms in split order (its own
-// from TMEM) and writes dW.  Called by the four epilogue warps between the cluster barriers.
-__device__ __forceinline__ int quarter_owner(int g, int splits) { return g * splits / 4; }
-
-__device__ __forceinline__ void cluster_send_quarter(uint32_t tmem_base, uint8_t* xchg, int g, int lane, int rank,
-                                                     int splits) {
-    const int owner = quarter_owner(g, splits);
-    const int slot = rank < owner ? rank : rank - 1;                 // the owner keeps no slot for itself
-    const int rows_owned = 128 / splits;
-    const int row_local = (g - owner * (4 / splits)) * 32 + lane;
-    const uint32_t local = ptx::smem_u32(xchg) + (uint32_t)((slot * rows_owned + row_local) * kXchgRowFloats) * 4u;
-    const uint32_t remote = ptx::map_shared_to_cta(local, (uint32_t)owner);
+// The tile's eight 32-column chunks are shared out among the CTAs (chunk ch belongs to CTA ch / (8 / splits)).
+// Every epilogue warp sends the chunks of its 32-row quarter that its CTA does not own from TMEM into the
+// owner's shared memory, and after a cluster barrier finishes the chunks its CTA owns: it adds the terms in
+// split order (its own from TMEM) and writes dW.  All four warps work in both phases.
+// Receive area of a CTA: [sender slot][128 rows][256 / splits columns + 4], fp32.
+__device__ __forceinline__ void cluster_send_chunks(uint32_t tmem_base, uint8_t* xchg, int g, int lane, int rank,
+                                                    int splits) {
+    const int cpo = (kBN / 32) / splits;                     // chunks per owner
+    const int pitch = cpo * 32 + 4;                          // floats per row of the receive area
+    const uint32_t row_off = (uint32_t)((32 * g + lane) * pitch) * 4u;
 #pragma unroll 1
     for (int ch = 0; ch < kBN / 32; ++ch) {
+        const int owner = ch / cpo;
+        if (owner == rank) continue;                         // uniform over the warp
+        const int slot = rank < owner ? rank : rank - 1;     // the owner keeps no slot for itself
+        const uint32_t local = ptx::smem_u32(xchg) + (uint32_t)(slot * kBM * pitch) * 4u + row_off +
+                               (uint32_t)((ch - owner * cpo) * 32) * 4u;
+        const uint32_t remote = ptx::map_shared_to_cta(local, (uint32_t)owner);
         uint32_t r[32];
         ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
         ptx::tmem_ld_wait();
 #pragma unroll
         for (int e = 0; e < 32; e += 4)
-            ptx::st_cluster_v4(remote + (uint32_t)(ch * 32 + e) * 4u, __uint_as_float(r[e]), __uint_as_float(r[e + 1]),
+            ptx::st_cluster_v4(remote + (uint32_t)e * 4u, __uint_as_float(r[e]), __uint_as_float(r[e + 1]),
                                __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
     }
 }
 
-__device__ __forceinline__ void cluster_finish_quarter(uint32_t tmem_base, const uint8_t* xchg, float* stage, int g,
-                                                       int lane, int rank, int splits, int j0, int c0, int Ca, int Cz,
-                                                       float* __restrict__ dw, int accumulate) {
-    const int rows_owned = 128 / splits;
-    const int row_local = (g - rank * (4 / splits)) * 32 + lane;
-    const float* mine = reinterpret_cast<const float*>(xchg) + (size_t)row_local * kXchgRowFloats;
+__device__ __forceinline__ void cluster_finish_chunks(uint32_t tmem_base, const uint8_t* xchg, float* stage, int g,
+                                                      int lane, int rank, int splits, int j0, int c0, int Ca, int Cz,
+                                                      float* __restrict__ dw, int accumulate) {
+    const int cpo = (kBN / 32) / splits;
+    const int pitch = cpo * 32 + 4;
+    const float* mine = reinterpret_cast<const float*>(xchg) + (size_t)(32 * g + lane) * pitch;
     const int rr0 = lane >> 3, q = lane & 7;
 #pragma unroll 1
-    for (int ch = 0; ch < kBN / 32; ++ch) {
+    for (int cl = 0; cl < cpo; ++cl) {
+        const int ch = rank * cpo + cl;
         uint32_t r[32];
         ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
         ptx::tmem_ld_wait();
@@ -271,7 +275,7 @@ __device__ __forceinline__ void cluster_finish_quarter(uint32_t tmem_base, const
                 for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(r[e]);
             } else {
                 const int slot = s < rank ? s : s - 1;
-                const float* src = mine + (size_t)slot * rows_owned * kXchgRowFloats + ch * 32;
+                const float* src = mine + (size_t)slot * kBM * pitch + cl * 32;
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
                     const float4 v = *reinterpret_cast<const float4*>(src + e);
@@ -456,12 +460,12 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         const int g = warp & 3;
         if (warp >= 2 && !*abort_flag) {
             ptx::tc_fence_after();
-            if (quarter_owner(g, splits) != split) cluster_send_quarter(tmem_base, xchg, g, lane, split, splits);
+            cluster_send_chunks(tmem_base, xchg, g, lane, split, splits);
         }
         __syncwarp();
-        ptx::cluster_sync_all();                                           // every quarter has been delivered
-        if (warp >= 2 && !*abort_flag && quarter_owner(g, splits) == split)
-            cluster_finish_quarter(tmem_base, xchg, stage, g, lane, split, splits, j0, c0, Ca, Cz, dw, accumulate);
+        ptx::cluster_sync_all();                                           // every chunk has been delivered
+        if (warp >= 2 && !*abort_flag)
+            cluster_finish_chunks(tmem_base, xchg, stage, g, lane, split, splits, j0, c0, Ca, Cz, dw, accumulate);
     }
 
     ptx::tc_fence_before();
