@@ -259,11 +259,11 @@ def run_ours(args, rank, world, device):
 # (weight_grad_gemm_wg_tc_kernel_vitb_fc1/fc2.txt, compress_fused_vitb_fc2.txt).  Set an entry to None
 # when its kernel changes, until the counters have been taken again.
 NCU_TRAFFIC = {
-    "wg_tc_kernel": 0.5 * ((96.870656e6 + 3.740160e6) + (96.890880e6 + 3.956480e6)),
+    "wg_tc_kernel": 0.5 * ((96.877056e6 + 4.115456e6) + (96.871424e6 + 4.160256e6)),
     "note_dw": "wg_tc_kernel alone (mean of fc1, fc2): dY 77.5 MB + dense scratch 19.4 MB read once; the decompress kernel "
-               "before it moves another 32.9 MB through DRAM on fc2 (13.8 read, 19.0 written, the rest of its 77.5 MB "
+               "before it moves another 33.0 MB through DRAM on fc2 (13.8 read, 19.2 written, the rest of its 77.5 MB "
                "output stays in L2 for the GEMM)",
-    "fused_compress_kernel_fc2": 78.055936e6 + 4.118528e6,
+    "fused_compress_kernel_fc2": 78.899712e6 + 3.401472e6,
 }
 
 
