@@ -1,10 +1,10 @@
 // bf16 min-k selection + packing as ONE persistent cooperative kernel (Sec. 3.3 "Min-K Elements",
 // Sec. 3.2 a-hat = {a_Xr, X_r}).
 //
-// Every WARP owns one contiguous run of 1024-element blocks and keeps it for the whole kernel, so
+// Every WARP owns one contiguous run of 512-element blocks and keeps it for the whole kernel, so
 // the ordered compaction needs no block-wide synchronisation and warps drift freely.
-//   sample  (separate 1-CTA kernel) a 16 Ki-element jittered sample brackets the threshold key T
-//           between two keys [lo, hi] (6-sigma margin on the sample rank); it also clears the selection state.
+//   sample  every CTA histograms the same 16 Ki-element jittered sample in shared memory and brackets
+//           the threshold key T between two keys [lo, hi] (6-sigma margin on the sample rank).
 //   phase 1 one read of the tensor: keys above hi are counted in a register, keys inside the band
 //           go to a small per-warp histogram, the rest is ignored (two packed bf16 per 32-bit word
 //           are classified with one add each, so the pass is bound by HBM, not by atomics).
@@ -14,10 +14,17 @@
 //           histograms.  No second counting pass.
 //   phase 3 second read (L2 hits for tensors that fit L2): element i is retained iff key_i > T, or
 //           key_i == T and fewer than q equal keys precede it; #retained before i =
-//           gt_before + min(eq_before, q).  Values are staged per warp and written in 16-byte pieces.
+//           gt_before + min(eq_before, q).  A lane owns 16 consecutive elements; retained values are
+//           staged per warp and leave in aligned 16-byte pieces.
 // When the band is wider than the per-warp histogram (small tensors, which are not sampled; key
 // distributions that are flat around T; a sample that missed) a general path is taken instead:
 // full CTA histogram in shared memory, global histogram by atomics, then one extra counting read.
+// Nothing in the scratch has to be cleared before a call: the grid barrier counts arrivals under a
+// number unique to the call, everything else is written before it is read.
+#include <unistd.h>
+
+#include <atomic>
+#include <chrono>
 #include <type_traits>
 
 #include "common.cuh"
@@ -26,7 +33,6 @@
 namespace dropit {
 
 constexpr int kFusedThreads = 1024;                             // main kernel; 1 CTA per SM
-constexpr int kSampleThreads = 1024;
 constexpr int kFusedWarps = kFusedThreads / 32;
 constexpr int kVpl = 2;                                        // 16-byte vectors per lane per warp block
 constexpr int kBlkVecs = 32 * kVpl;                            // vectors per warp block
@@ -43,13 +49,15 @@ constexpr uint32_t kHiBits = 0x80008000u;
 constexpr int kRingDepth = 4;                                  // blocks of a warp's run in flight (cp.async ring)
 constexpr int kRingSlotBytes = kBlkVecs * 16;                  // one block
 constexpr size_t kRingBytes = (size_t)kFusedWarps * kRingDepth * kRingSlotBytes;   // 128 KB
-constexpr int kStageVals = kBlkElems + 16;                     // per-warp staging, values
-constexpr int kStageIdx = kBlkElems + 8;                       // per-warp staging, indices
+constexpr int kStageCap = 1024;                                // per-warp circular staging of retained values (power of two)
+constexpr int kFlushVals = 256;                                // staged values that trigger a flush: one 16-byte piece per lane
+static_assert(kFlushVals + kBlkElems + 8 <= kStageCap, "a block must fit behind what a flush leaves");
+constexpr size_t kStageBytes = (size_t)kFusedWarps * kStageCap * 2;   // 64 KB
+static_assert(kStageBytes >= (size_t)kKeySpace * 2, "the sample's 16-bit histogram lives in the staging area");
 
 struct FusedState {
-    uint32_t barrier;            // grid-barrier arrivals
-    uint32_t band_lo, band_hi;   // written by the sample kernel
-    uint32_t pad0;
+    unsigned long long barrier;  // grid barrier: call epoch << 32 | arrivals (needs no clearing between calls)
+    uint32_t pad0[2];
     unsigned long long n_hi[2];  // general path: #{key > hi} per attempt
     uint32_t reserved[24];
 };
@@ -59,7 +67,7 @@ struct FusedPlan {
     int64_t blocks_total;
     int grid;
     int blocks_per_warp;
-    size_t hist_off[2], agg_off, rows_off, total_bytes, zero_bytes;
+    size_t hist_off[2], agg_off, rows_off, total_bytes;
 };
 
 static FusedPlan make_fused_plan(int64_t n) {
@@ -76,13 +84,23 @@ static FusedPlan make_fused_plan(int64_t n) {
     p.hist_off[0] = kStateBytes;
     p.hist_off[1] = p.hist_off[0] + (size_t)kKeySpace * 4;
     p.agg_off = p.hist_off[1] + (size_t)kKeySpace * 4;
-    p.zero_bytes = kStateBytes;                                 // the rest is written before it is read
     p.rows_off = p.agg_off + (size_t)kMaxGrid * 8;
     p.total_bytes = p.rows_off + (size_t)kMaxGrid * kRowWords * 4;
     return p;
 }
 
 size_t fused_compress_workspace_bytes(int64_t n) { return make_fused_plan(n).total_bytes; }
+
+// A number that no earlier call of this process has used (and that another process is unlikely to
+// have left in recycled memory): the grid barrier tells its own arrivals from stale ones by it.
+static uint32_t next_epoch() {
+    static std::atomic<uint32_t> counter{[] {
+        const uint64_t t = (uint64_t)std::chrono::steady_clock::now().time_since_epoch().count();
+        uint64_t h = (t ^ ((uint64_t)getpid() << 32)) * 0x9E3779B97F4A7C15ull;
+        return (uint32_t)(h >> 32);
+    }()};
+    return counter.fetch_add(1u, std::memory_order_relaxed);
+}
 
 __device__ __forceinline__ uint32_t ptx_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -112,6 +130,15 @@ __device__ __forceinline__ uint32_t flags4(uint32_t x, uint32_t y) {
     return ((t * 0x00204081u) >> 21) & 0xFu;
 }
 
+// Eight flags held in bit 15 and bit 31 of four words -> 8 bits in element order.  prmt gathers the flag
+// bytes of each pair of words; flags of the first pair go to bit 0 of each byte, of the second pair to
+// bit 4; one multiply lines all eight up at bits 24..31 (no two partial products share a bit, so no carries).
+__device__ __forceinline__ uint32_t flags8(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3) {
+    const uint32_t r0 = __byte_perm(x0, x1, 0x7531), r1 = __byte_perm(x2, x3, 0x7531);
+    const uint32_t u = ((r0 >> 7) & 0x01010101u) | ((r1 >> 3) & 0x10101010u);
+    return (u * 0x01020408u) >> 24;
+}
+
 // Exclusive prefix over the block's threads of `v`; also returns the block total.
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s_warp, uint32_t* total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -136,97 +163,6 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
     return wprefix + inc - v;
 }
 
-// ---------------------------------------------------------------------------------------------
-// Sample kernel: zero the scratch, bracket the threshold key.
-// ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kSampleThreads, 1)
-sample_band_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long k, unsigned char* ws, size_t zero_bytes) {
-    extern __shared__ uint32_t bins[];
-    __shared__ uint32_t s_warp[32];
-    __shared__ uint32_t s_band[2];
-#ifdef DROPIT_PHASE_TIMING
-    unsigned long long t_begin;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_begin));
-#endif
-    ptx::grid_dependency_wait();   // launched programmatically: x may come from the kernel before this one
-    const int64_t nvec = n / 8;
-    const bool sampled = n >= kSampleMinElems;
-    uint4 sv[kSampleVecs / kSampleThreads];
-    if (sampled) {   // issue the sample loads first; they fly while the scratch is zeroed
-        const int64_t stride = nvec / kSampleVecs;   // >= 32
-#pragma unroll
-        for (int r = 0; r < kSampleVecs / kSampleThreads; ++r) {
-            const uint32_t s = r * kSampleThreads + threadIdx.x;
-            const uint32_t h = (s * 2654435761u) >> 7;   // jitter inside the stride window
-            sv[r] = ld_stream(x + (int64_t)s * stride + (int64_t)(h % (uint32_t)stride));
-        }
-    }
-    uint4* z = reinterpret_cast<uint4*>(ws);
-    for (size_t i = threadIdx.x; i < zero_bytes / 16; i += blockDim.x) z[i] = make_uint4(0, 0, 0, 0);
-    FusedState* st = reinterpret_cast<FusedState*>(ws);
-    if (threadIdx.x == 0) {
-        s_band[0] = 0;
-        s_band[1] = kKeySpace - 1;
-    }
-    if (sampled) {
-        for (int i = threadIdx.x; i < kKeySpace; i += blockDim.x) bins[i] = 0;
-        __syncthreads();
-#pragma unroll
-        for (int r = 0; r < kSampleVecs / kSampleThreads; ++r) {
-            uint32_t key[8];
-            keys_of(sv[r], key);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) atomicAdd(&bins[key[e]], 1u);
-        }
-        __syncthreads();
-        // ranks (counted from the largest key) that bracket the threshold with a 6-sigma margin
-        const float S = (float)(kSampleVecs * 8);
-        const float p = (float)((double)k / (double)n);
-        const float ks = p * S;
-        const float margin = 6.0f * sqrtf(S * p * (1.0f - p)) + 16.0f;
-        const float r_hi = ks - margin, r_lo = ks + margin;
-        constexpr int PER = kKeySpace / kSampleThreads;
-        const int t = threadIdx.x;
-        uint32_t sum = 0;
-#pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            // rotate the start so that the 32 lanes of a warp hit 32 different banks
-            const int rr = (r + t) & (PER - 1);
-            sum += bins[kKeySpace - 1 - (t * PER + rr)];
-        }
-        uint32_t total;
-        const uint32_t excl = block_exclusive_scan(sum, s_warp, &total);
-        // key at descending rank r: cum_before < r <= cum_before + h
-        if ((r_hi >= 1.0f && (float)excl < r_hi && r_hi <= (float)(excl + sum)) ||
-            (r_lo <= S && (float)excl < r_lo && r_lo <= (float)(excl + sum))) {
-            uint32_t cum = excl;
-            for (int r = 0; r < PER; ++r) {
-                const uint32_t key = kKeySpace - 1 - (t * PER + r);
-                const uint32_t hh = bins[key];
-                if (hh) {
-                    if (r_hi >= 1.0f && (float)cum < r_hi && r_hi <= (float)(cum + hh)) s_band[1] = key;
-                    if (r_lo <= S && (float)cum < r_lo && r_lo <= (float)(cum + hh)) s_band[0] = key;
-                }
-                cum += hh;
-            }
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        st->band_lo = s_band[0];
-        st->band_hi = s_band[1];
-#ifdef DROPIT_PHASE_TIMING
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        reinterpret_cast<unsigned long long*>(st->reserved)[6] = t;
-        reinterpret_cast<unsigned long long*>(st->reserved)[7] = t_begin;
-#endif
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Main kernel.
-// ---------------------------------------------------------------------------------------------
 // Optional phase timestamps of CTA 0 (build with -DDROPIT_PHASE_TIMING): FusedState::reserved holds
 // %globaltimer at each stamp.  Off in normal builds.
 #ifdef DROPIT_PHASE_TIMING
@@ -241,6 +177,90 @@ __device__ __forceinline__ void phase_stamp(FusedState* st, int i) {
 __device__ __forceinline__ void phase_stamp(FusedState*, int) {}
 #endif
 
+// ---------------------------------------------------------------------------------------------
+// Sample step: bracket the threshold key.  Every CTA runs it on the same 16 Ki elements (the first
+// CTA to ask brings them in from HBM, the others read them from L2) and therefore arrives at the
+// same band without any exchange.  `bins`: kKeySpace counters in shared memory; band[0..1] = lo, hi.
+// Ends with a block-wide barrier.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t sample_count(const uint32_t* bins, uint32_t key) {
+    return (bins[key >> 1] >> ((key & 1u) * 16)) & 0xFFFFu;
+}
+
+template <typename AfterLoads>
+__device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t n, unsigned long long k, uint32_t* bins,
+                                            uint32_t* s_warp, uint32_t* band, FusedState* st, AfterLoads after_loads) {
+    const int64_t nvec = n / 8;
+    const bool sampled = n >= kSampleMinElems;
+    uint4 sv[kSampleVecs / kFusedThreads];
+    if (sampled) {   // issue the sample loads first; they fly while the counters are cleared
+        const int64_t stride = nvec / kSampleVecs;   // >= 32
+#pragma unroll
+        for (int r = 0; r < kSampleVecs / kFusedThreads; ++r) {
+            const uint32_t s = r * kFusedThreads + threadIdx.x;
+            const uint32_t h = (s * 2654435761u) >> 7;   // jitter inside the stride window
+            sv[r] = ld_stream(x + (int64_t)s * stride + (int64_t)(h % (uint32_t)stride));
+        }
+    }
+    after_loads();   // whatever the caller wants in flight behind the sample loads
+    if (threadIdx.x == 0) {
+        band[0] = 0;
+        band[1] = kKeySpace - 1;
+    }
+    if (sampled) {
+        // two 16-bit counters per word (a counter holds at most the sample size, 16384)
+        uint4* z = reinterpret_cast<uint4*>(bins);
+        for (int i = threadIdx.x; i < kKeySpace / 8; i += kFusedThreads) z[i] = make_uint4(0, 0, 0, 0);
+        __syncthreads();
+        phase_stamp(st, 8);
+#pragma unroll
+        for (int r = 0; r < kSampleVecs / kFusedThreads; ++r) {
+            uint32_t key[8];
+            keys_of(sv[r], key);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) atomicAdd(&bins[key[e] >> 1], 1u << ((key[e] & 1u) * 16));
+        }
+        __syncthreads();
+        phase_stamp(st, 9);
+        // ranks (counted from the largest key) that bracket the threshold with a 6-sigma margin
+        const float S = (float)(kSampleVecs * 8);
+        const float p = (float)((double)k / (double)n);
+        const float ks = p * S;
+        const float margin = 6.0f * sqrtf(S * p * (1.0f - p)) + 16.0f;
+        const float r_hi = ks - margin, r_lo = ks + margin;
+        constexpr int PER = kKeySpace / kFusedThreads;   // keys per thread, descending: kKeySpace-1 - (t*PER + r)
+        const int t = threadIdx.x;
+        const uint32_t* mine = bins + (kKeySpace / 2 - (t + 1) * (PER / 2));   // the thread's PER/2 words
+        uint32_t sum = 0;
+#pragma unroll
+        for (int r = 0; r < PER / 2; ++r) {
+            const uint32_t w = mine[(r + t) & (PER / 2 - 1)];   // rotated start: fewer bank conflicts
+            sum += (w & 0xFFFFu) + (w >> 16);
+        }
+        uint32_t total;
+        const uint32_t excl = block_exclusive_scan(sum, s_warp, &total);
+        phase_stamp(st, 10);
+        // key at descending rank r: cum_before < r <= cum_before + h
+        if ((r_hi >= 1.0f && (float)excl < r_hi && r_hi <= (float)(excl + sum)) ||
+            (r_lo <= S && (float)excl < r_lo && r_lo <= (float)(excl + sum))) {
+            uint32_t cum = excl;
+            for (int r = 0; r < PER; ++r) {
+                const uint32_t key = kKeySpace - 1 - (t * PER + r);
+                const uint32_t hh = sample_count(bins, key);
+                if (hh) {
+                    if (r_hi >= 1.0f && (float)cum < r_hi && r_hi <= (float)(cum + hh)) band[1] = key;
+                    if (r_lo <= S && (float)cum < r_lo && r_lo <= (float)(cum + hh)) band[0] = key;
+                }
+                cum += hh;
+            }
+        }
+    }
+    __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Main kernel.
+// ---------------------------------------------------------------------------------------------
 struct FusedShared {
     uint32_t warp[32];
     unsigned long long red64[32];
@@ -250,20 +270,43 @@ struct FusedShared {
     uint32_t pre[kRowWords];                  // ... over the CTAs before this one
     uint32_t wpre_gt[kFusedWarps], wpre_eq[kFusedWarps];   // exclusive prefix of each warp (absolute)
     uint32_t T, found;
+    uint32_t band[2];                         // lo, hi from the sample
     unsigned long long n_gt, quota;
     int ok;
 };
 
-__device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target, int* s_ok) {
+// Grid barrier on one 64-bit word = (epoch << 32 | arrivals).  `epoch` is unique to the call; CTA 0
+// stores (epoch << 32) into the word when the kernel starts (barrier_open), so nothing has to be cleared
+// between calls or before the first one.  An arriving CTA waits until the word carries its epoch (it
+// does, long since, in any normal run), adds one, and waits for `target` = the arrivals expected so far
+// in this call.  Every wait is bounded: returns false when one runs out.
+__device__ __forceinline__ void barrier_open(unsigned long long* word, uint32_t epoch) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(word), "l"((unsigned long long)epoch << 32) : "memory");
+    }
+}
+__device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t epoch, uint32_t target, int* s_ok) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        atomicAdd(counter, 1u);
-        int spins = 0;
         bool ok = true;
-        while (ld_acquire_u32(counter) < target) {
+        int spins = 0;
+        unsigned long long v;
+        for (;;) {   // the word belongs to this call
+            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(word) : "memory");
+            if ((uint32_t)(v >> 32) == epoch) break;
             if (++spins > kBarrierSpinLimit) { ok = false; break; }
             __nanosleep(32);
+        }
+        if (ok) {
+            atomicAdd(word, 1ull);
+            const unsigned long long goal = ((unsigned long long)epoch << 32) | target;
+            for (;;) {
+                asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(word) : "memory");
+                if (v >= goal) break;
+                if (++spins > kBarrierSpinLimit) { ok = false; break; }
+                __nanosleep(32);
+            }
         }
         __threadfence();
         *s_ok = ok ? 1 : 0;
@@ -361,45 +404,20 @@ __device__ __forceinline__ int valid_elems(int64_t vi, int64_t nvec_full, int64_
     return vi < nvec_full ? 8 : (vi == nvec_full ? (int)(n & 7) : 0);
 }
 
-// Write the whole 16-byte pieces of a warp's staging buffer and carry the remainder to its front.
-// Slot s of the buffer maps to out[base + s] with base a multiple of PIECE elements; the first
-// `foreign` slots of the very first piece belong to the previous warp and are never written.
-template <typename E, int PIECE>
-__device__ __forceinline__ void flush_pieces(E* stage, E* out_base, uint32_t kept, uint32_t& pend, uint32_t& foreign,
-                                             int lane) {
-    const uint32_t total = pend + kept;
-    const uint32_t nfull = total / PIECE;
-    uint32_t c0 = 0;
-    if (foreign && nfull > 0) {
-        if (lane >= (int)foreign && lane < PIECE) out_base[lane] = stage[lane];
-        c0 = 1;
-        foreign = 0;
-    }
-    for (uint32_t c = c0 + lane; c < nfull; c += 32)
-        reinterpret_cast<uint4*>(out_base)[c] = reinterpret_cast<const uint4*>(stage)[c];
-    const uint32_t rem = total - nfull * PIECE;
-    E carry = 0;
-    if (nfull > 0 && lane < (int)rem) carry = stage[nfull * PIECE + lane];
-    __syncwarp();
-    if (nfull > 0 && lane < (int)rem) stage[lane] = carry;
-    pend = rem;   // == total when nfull == 0
-    __syncwarp();
-}
-
 template <bool INDEX32>
 __global__ void __launch_bounds__(kFusedThreads, 1)
-fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long k, int blocks_per_warp,
+fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long k, int blocks_per_warp, uint32_t epoch,
                       unsigned char* ws, size_t hist_off0, size_t hist_off1, size_t agg_off, size_t rows_off,
                       uint16_t* __restrict__ values, uint32_t* __restrict__ mask, int32_t* __restrict__ indices,
                       uint32_t* __restrict__ offsets, int32_t* dev_status) {
+    // shared memory: [input ring, 128 KB | general path: full key histogram]
+    //                [phase 3: per-warp value staging, 64 KB | sample step: 16-bit key histogram]
+    //                [control block of phases 1-2]
     extern __shared__ __align__(16) unsigned char fsm[];
-    uint32_t* bins = reinterpret_cast<uint32_t*>(fsm);   // general path, phases 1-2: kKeySpace counters
-    // phases 1-2 keep their control block where phase 3 later stages values (phase 3 needs no control block)
-    FusedShared& sh = *reinterpret_cast<FusedShared*>(fsm + kRingBytes);
-    static_assert(sizeof(FusedShared) <= (size_t)kFusedWarps * kStageVals * 2, "control block must fit the staging area");
-    // the input ring shares its memory with the general path's histogram (never live together)
-    uint16_t* s_vals_all = reinterpret_cast<uint16_t*>(fsm + kRingBytes);   // phase 3: per-warp staging
-    int32_t* s_idx_all = reinterpret_cast<int32_t*>(fsm + kRingBytes + (size_t)kFusedWarps * kStageVals * 2);
+    uint32_t* bins = reinterpret_cast<uint32_t*>(fsm);
+    uint32_t* sample_bins = reinterpret_cast<uint32_t*>(fsm + kRingBytes);
+    uint16_t* s_vals_all = reinterpret_cast<uint16_t*>(fsm + kRingBytes);
+    FusedShared& sh = *reinterpret_cast<FusedShared*>(fsm + kRingBytes + kStageBytes);
 
     FusedState* st = reinterpret_cast<FusedState*>(ws);
     unsigned long long* agg = reinterpret_cast<unsigned long long*>(ws + agg_off);
@@ -420,7 +438,20 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     };
     uint32_t barrier_target = 0;
 
-    uint32_t lo = st->band_lo, hi = st->band_hi;
+    phase_stamp(st, 7);
+    // the general path's totals start at zero; the grid barriers order this store before their first use
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        st->n_hi[0] = 0;
+        st->n_hi[1] = 0;
+    }
+    barrier_open(&st->barrier, epoch);
+    // the first blocks of the run are requested right behind the sample loads, whose processing hides their latency
+    bool prefetched = true;
+    sample_band(x, n, k, sample_bins, sh.warp, sh.band, st, [&] {
+#pragma unroll
+        for (int d = 0; d < kRingDepth - 1; ++d) issue_block(blk0 + d, ring_lane + d * kRingSlotBytes);
+    });
+    uint32_t lo = sh.band[0], hi = sh.band[1];
     uint32_t T = 0, q = 0;
     uint32_t run_gt = 0, run_eq = 0;   // this warp's exclusive prefix (absolute)
     phase_stamp(st, 0);
@@ -437,6 +468,10 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         if (narrow) {
             for (int i = threadIdx.x; i < kFusedWarps * kWarpBins; i += blockDim.x) (&sh.whist[0][0])[i] = 0;
         } else {
+            if (prefetched) {   // the histogram takes the ring's memory: let the requested blocks land first
+                asm volatile("cp.async.wait_all;" ::: "memory");
+                __syncthreads();
+            }
             for (uint32_t i = threadIdx.x; i <= width; i += blockDim.x) bins[i] = 0;
         }
         __syncthreads();
@@ -473,8 +508,10 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         };
         if (narrow) {
             // stream the run through the ring, kRingDepth-1 blocks ahead
+            if (!prefetched) {
 #pragma unroll
-            for (int d = 0; d < kRingDepth - 1; ++d) issue_block(blk0 + d, ring_lane + d * kRingSlotBytes);
+                for (int d = 0; d < kRingDepth - 1; ++d) issue_block(blk0 + d, ring_lane + d * kRingSlotBytes);
+            }
             int slot = 0, slot_ahead = kRingDepth - 1;
             for (int64_t blk = blk0; blk < blk1; ++blk) {
                 issue_block(blk + kRingDepth - 1, ring_lane + slot_ahead * kRingSlotBytes);
@@ -513,6 +550,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                 for (int j = 0; j < kVpl; ++j) count_vec(va[j], na[j]);
             }
         }
+        prefetched = false;
         phase_stamp(st, 1);
         for (int o = 16; o > 0; o >>= 1) {
             cnt_lo += __shfl_xor_sync(kFullMask, cnt_lo, o);
@@ -541,7 +579,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             // grid barrier separates the clearing from the accumulation
             for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i <= width; i += gridDim.x * blockDim.x) ghist[i] = 0;
             barrier_target += gridDim.x;
-            if (!grid_barrier(&st->barrier, barrier_target, &sh.ok)) {
+            if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok)) {
                 if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
                 return;
             }
@@ -552,7 +590,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             if (threadIdx.x == 0 && cta_hi) atomicAdd(&st->n_hi[attempt], (unsigned long long)cta_hi);
         }
         barrier_target += gridDim.x;
-        if (!grid_barrier(&st->barrier, barrier_target, &sh.ok)) {
+        if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok)) {
             if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
             return;
         }
@@ -568,40 +606,57 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             }
             __syncthreads();
             {
-                const uint32_t ncol = width + 2;   // bins 0..width, then #key>hi (stored at kWarpBins)
-                const uint32_t cells = gridDim.x * ncol;
-                for (uint32_t i0 = threadIdx.x; i0 < cells; i0 += 4 * blockDim.x) {
-                    uint32_t val[4], col[4], row[4];
+                // thread (g, c) adds column c of rows g, g + kGroups, ...: consecutive threads read consecutive
+                // words of a row, and a thread's loads are independent of one another
+                constexpr int kGroups = kFusedThreads / kRowWords;
+                constexpr int kInFlight = 8;
+                const uint32_t g = threadIdx.x / kRowWords, c = threadIdx.x - g * kRowWords;
+                if (g < (uint32_t)kGroups && (c <= width || c == (uint32_t)kWarpBins)) {
+                    uint32_t t_sum = 0, p_sum = 0;
+                    for (uint32_t r0 = g; r0 < gridDim.x; r0 += kInFlight * kGroups) {
+                        uint32_t val[kInFlight];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const uint32_t i = i0 + u * blockDim.x;
-                        row[u] = i / ncol;
-                        const uint32_t c = i - row[u] * ncol;
-                        col[u] = (c == width + 1) ? (uint32_t)kWarpBins : c;
-                        val[u] = (i < cells) ? __ldcg(&rows[(size_t)row[u] * kRowWords + col[u]]) : 0u;
-                    }
+                        for (int u = 0; u < kInFlight; ++u) {
+                            const uint32_t r = r0 + u * kGroups;
+                            val[u] = (r < gridDim.x) ? __ldcg(&rows[(size_t)r * kRowWords + c]) : 0u;
+                        }
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (val[u]) {
-                            atomicAdd(&sh.tot[col[u]], val[u]);
-                            if (row[u] < blockIdx.x) atomicAdd(&sh.pre[col[u]], val[u]);
+                        for (int u = 0; u < kInFlight; ++u) {
+                            t_sum += val[u];
+                            if (r0 + u * kGroups < blockIdx.x) p_sum += val[u];
                         }
                     }
+                    if (t_sum) atomicAdd(&sh.tot[c], t_sum);
+                    if (p_sum) atomicAdd(&sh.pre[c], p_sum);
                 }
             }
             __syncthreads();
-            if (threadIdx.x == 0) {
-                unsigned long long cum = sh.tot[kWarpBins];   // keys above the band
-                for (int d = (int)width; d >= 0; --d) {
-                    const uint32_t hcount = sh.tot[d];
-                    if (cum < k && k <= cum + hcount) {
-                        sh.T = lo + d;
+            if (warp == 0) {
+                // bins in descending key order, two per lane: the bin that takes the running count past k is T
+                const unsigned long long above = sh.tot[kWarpBins];   // keys above the band
+                uint32_t h[2], inc[2];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const uint32_t pos = j * 32 + lane;
+                    h[j] = (pos <= width) ? sh.tot[width - pos] : 0u;
+                    inc[j] = h[j];
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t y = __shfl_up_sync(kFullMask, inc[j], o);
+                        if (lane >= o) inc[j] += y;
+                    }
+                }
+                inc[1] += __shfl_sync(kFullMask, inc[0], 31);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const uint32_t pos = j * 32 + lane;
+                    const unsigned long long cum = above + (inc[j] - h[j]);
+                    if (pos <= width && cum < k && k <= cum + h[j]) {
+                        sh.T = lo + (width - pos);
                         sh.n_gt = cum;
                         sh.quota = k - cum;
                         sh.found = 1;
-                        break;
                     }
-                    cum += hcount;
                 }
             }
             __syncthreads();
@@ -609,30 +664,34 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             T = sh.T;
             q = (uint32_t)sh.quota;
             const uint32_t dT = T - lo;
-            if (warp == 0) {
-                // lane = warp index: that warp's (gt, eq), then an exclusive scan over the 32 warps
-                uint32_t g = 0, e = 0;
-                if (lane < kFusedWarps) {
-                    g = sh.w_hi[lane];
-                    e = sh.whist[lane][dT];
-                    for (uint32_t d = dT + 1; d <= width; ++d) g += sh.whist[lane][d];
+            {
+                // this warp's (#key > T, #key == T) and the same over the CTAs before this one
+                uint32_t g = 0, pg = 0;
+                for (uint32_t d = dT + 1 + lane; d <= width; d += 32) {
+                    g += sh.whist[warp][d];
+                    pg += sh.pre[d];
                 }
-                uint32_t gi = g, ei = e;
+                for (int o = 16; o > 0; o >>= 1) {
+                    g += __shfl_xor_sync(kFullMask, g, o);
+                    pg += __shfl_xor_sync(kFullMask, pg, o);
+                }
+                if (lane == 0) {
+                    sh.wpre_gt[warp] = g + sh.w_hi[warp];
+                    sh.wpre_eq[warp] = sh.whist[warp][dT];
+                }
+                __syncthreads();
+                // exclusive scan over the CTA's warps (lane = warp index), done by every warp for itself
+                const uint32_t og = (lane < kFusedWarps) ? sh.wpre_gt[lane] : 0u;
+                const uint32_t oe = (lane < kFusedWarps) ? sh.wpre_eq[lane] : 0u;
+                uint32_t gi = og, ei = oe;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const uint32_t yg = __shfl_up_sync(kFullMask, gi, o), ye = __shfl_up_sync(kFullMask, ei, o);
                     if (lane >= o) { gi += yg; ei += ye; }
                 }
-                uint32_t cta_pre_gt = sh.pre[kWarpBins], cta_pre_eq = sh.pre[dT];
-                for (uint32_t d = dT + 1; d <= width; ++d) cta_pre_gt += sh.pre[d];
-                if (lane < kFusedWarps) {
-                    sh.wpre_gt[lane] = cta_pre_gt + gi - g;
-                    sh.wpre_eq[lane] = cta_pre_eq + ei - e;
-                }
+                run_gt = pg + sh.pre[kWarpBins] + __shfl_sync(kFullMask, gi - og, warp);
+                run_eq = sh.pre[dT] + __shfl_sync(kFullMask, ei - oe, warp);
             }
-            __syncthreads();
-            run_gt = sh.wpre_gt[warp];
-            run_eq = sh.wpre_eq[warp];
             break;
         }
         // ---- general path: T from the global histogram ----
@@ -709,7 +768,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             }
             if (threadIdx.x == 0) st_relaxed_u64(&agg[blockIdx.x], ((unsigned long long)ce << 32) | cg);
             barrier_target += gridDim.x;
-            if (!grid_barrier(&st->barrier, barrier_target, &sh.ok)) {
+            if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok)) {
                 if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
                 return;
             }
@@ -728,148 +787,152 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     phase_stamp(st, 3);
 
     // ---------------- phase 3: ordered compaction, one warp per run of blocks ----------------
+    // A lane owns 16 CONSECUTIVE elements of a block (vectors 2*lane and 2*lane+1), i.e. half a mask
+    // word, so a block costs one warp scan and one shuffle for the mask.  The copies into the ring
+    // stay coalesced (lane copies vectors lane and lane+32); vector v sits at 16-byte position
+    // v ^ ((v >> 3) & 1) of its slot so that neither side has bank conflicts.  Retained values go to
+    // a per-warp circular buffer indexed by their final position in `values` (mod kStageCap) and
+    // leave for global memory as one aligned 16-byte piece per lane once kFlushVals are staged.
     ptx::launch_dependents();   // a programmatically launched kernel behind this one may be brought up
     const int64_t nwords = (n + 31) / 32;
-    uint16_t* s_vals = s_vals_all + (size_t)warp * kStageVals;
-    int32_t* s_idx = s_idx_all + (size_t)warp * kStageIdx;
+    uint16_t* s_vals = s_vals_all + (size_t)warp * kStageCap;
+    const uint32_t s_vals_addr = ptx_smem(s_vals);
     const uint32_t c_gt = ge_const(T + 1), c_ge = ge_const(T);
+    const uint32_t ring_warp = ptx_smem(fsm) + (warp * kRingDepth) * kRingSlotBytes;
+    const uint32_t ring_copy = ring_warp + ((lane ^ ((lane >> 3) & 1)) * 16);   // where vector `lane` of a slot goes
+    const uint32_t swz = (lane >> 2) & 1;                                        // swizzle bit of vectors 2*lane, 2*lane+1
+    const uint32_t ring_own = ring_warp + lane * 32;                             // the lane's 32 bytes of a slot
+    auto issue3 = [&](int64_t b, uint32_t dst) {
+        if (b < blk_full_end) ring_issue_full(dst, x + b * kBlkVecs + lane);
+        else if (b < blk1) ring_issue(dst, x, b, lane, nvec_full, n);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    };
     uint32_t gpos = run_gt + min(run_eq, q);   // retained elements before this warp's next block
-    uint32_t pend = gpos & 7u, foreign = pend;       // staged-but-unwritten values; leading slots not ours
-    uint32_t pend_i = gpos & 3u, foreign_i = pend_i;
+    uint32_t head = gpos & ~7u;                // first position not yet written to `values` (16-byte aligned)
+    uint32_t foreign = gpos & 7u;              // leading slots of the first piece that belong to the previous warp
+    // Write staged positions [head, head + 8 * pieces): piece c by lane c % 32.
+    auto flush = [&](uint32_t pieces) {
+        for (uint32_t c = lane; c < pieces; c += 32) {
+            const uint32_t p = head + c * 8;
+            if (c == 0 && foreign) {
+                for (uint32_t e = foreign; e < 8; ++e) values[p + e] = s_vals[(p + e) & (kStageCap - 1)];
+            } else {
+                *reinterpret_cast<uint4*>(values + p) = *reinterpret_cast<const uint4*>(s_vals + (p & (kStageCap - 1)));
+            }
+        }
+        if (pieces) foreign = 0;
+        head += pieces * 8;
+        __syncwarp();   // the slots may be staged again only after every lane has read its piece
+    };
 #pragma unroll
-    for (int d = 0; d < kRingDepth - 1; ++d) issue_block(blk0 + d, ring_lane + d * kRingSlotBytes);
+    for (int d = 0; d < kRingDepth - 1; ++d) issue3(blk0 + d, ring_copy + d * kRingSlotBytes);
     int slot = 0, slot_ahead = kRingDepth - 1;
     // One block of the run.  FULL: every vector of the block is whole, so the bounds arithmetic folds away.
     auto compact_block = [&](int64_t blk, auto full_tag) {
         constexpr bool FULL = decltype(full_tag)::value;
-        issue_block(blk + kRingDepth - 1, ring_lane + slot_ahead * kRingSlotBytes);
+        issue3(blk + kRingDepth - 1, ring_copy + slot_ahead * kRingSlotBytes);
         ring_wait();
-        uint4 cur[kVpl];
-        ring_read(ring_lane + slot * kRingSlotBytes, cur);
+        __syncwarp();   // the lane reads vectors that other lanes copied
+        const uint32_t own = ring_own + slot * kRingSlotBytes;
+        uint32_t w[8];
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(own + swz * 16) : "memory");
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(own + (swz ^ 1u) * 16) : "memory");
         slot = (slot + 1 == kRingDepth) ? 0 : slot + 1;
         slot_ahead = (slot_ahead + 1 == kRingDepth) ? 0 : slot_ahead + 1;
-        uint32_t gt8[kVpl], eq8[kVpl], cnt[kVpl];
+        uint32_t a[8], eany = 0;
 #pragma unroll
-        for (int j = 0; j < kVpl; ++j) {
-            const uint32_t w[4] = {cur[j].x, cur[j].y, cur[j].z, cur[j].w};
-            uint32_t a[4], eb[4], eany = 0;
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t m = w[i] & 0x7FFF7FFFu;
+            a[i] = m + c_gt;                        // bit 15 of a half: key > T
+            eany |= (m + c_ge) & ~a[i];             // bit 15 of a half: key == T
+        }
+        const uint32_t g16 = flags8(a[0], a[1], a[2], a[3]) | (flags8(a[4], a[5], a[6], a[7]) << 8);
+        uint32_t e16 = 0;
+        if (eany & kHiBits) {
+            uint32_t eb[8];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t m = w[i] & 0x7FFF7FFFu;
-                a[i] = m + c_gt;                        // bit 15 of a half: key > T
-                eb[i] = (m + c_ge) & ~a[i];             // bit 15 of a half: key == T
-                eany |= eb[i];
+            for (int i = 0; i < 8; ++i) eb[i] = ((w[i] & 0x7FFF7FFFu) + c_ge) & ~a[i];
+            e16 = flags8(eb[0], eb[1], eb[2], eb[3]) | (flags8(eb[4], eb[5], eb[6], eb[7]) << 8);
+            if constexpr (!FULL) {   // zero padding past the end must not tie with T = 0
+                const int64_t left = n - (blk * kBlkElems + lane * 16);
+                e16 &= left >= 16 ? 0xFFFFu : (left > 0 ? (1u << (int)left) - 1u : 0u);
             }
-            const uint32_t g8 = flags4(a[0], a[1]) | (flags4(a[2], a[3]) << 4);
-            uint32_t e8 = 0;
-            if (eany & kHiBits) {
-                e8 = flags4(eb[0], eb[1]) | (flags4(eb[2], eb[3]) << 4);
-                if constexpr (!FULL) {   // zero padding past the end must not tie with T = 0
-                    const int nvalid = valid_elems(blk * kBlkVecs + j * 32 + lane, nvec_full, n);
-                    e8 &= (1u << nvalid) - 1u;
+        }
+        const uint32_t cnt = __popc(g16) | (__popc(e16) << 16);
+        // packed (gt | eq << 16) prefix over the lanes = over the block's elements
+        uint32_t inc = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(kFullMask, inc, o);
+            if (lane >= o) inc += y;
+        }
+        const uint32_t tot = __shfl_sync(kFullMask, inc, 31);
+        const uint32_t excl = inc - cnt;
+        const uint32_t eq_before = run_eq + (excl >> 16);
+        uint32_t keep = g16;
+        if (e16) {
+            const uint32_t room = (eq_before < q) ? (q - eq_before) : 0u;
+            uint32_t ke = e16;
+            if (room < (cnt >> 16)) {   // the quota ends inside this lane's ties: the first `room` of them stay
+                uint32_t m = e16;
+                ke = 0;
+                for (uint32_t r = 0; r < room; ++r) {
+                    ke |= m & (0u - m);
+                    m &= m - 1;
                 }
             }
-            gt8[j] = g8;
-            eq8[j] = e8;
-            cnt[j] = __popc(g8) | (__popc(e8) << 16);
+            keep |= ke;
         }
-
-        // packed (gt | eq << 16) prefix inside the warp in (j, lane) order
-        uint32_t excl[kVpl];
-        uint32_t row_base = 0;
-#pragma unroll
-        for (int j = 0; j < kVpl; ++j) {
-            uint32_t inc = cnt[j];
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t y = __shfl_up_sync(kFullMask, inc, o);
-                if (lane >= o) inc += y;
-            }
-            excl[j] = row_base + inc - cnt[j];
-            row_base += __shfl_sync(kFullMask, inc, 31);
-        }
-        const uint32_t blk_gt = row_base & 0xFFFFu, blk_eq = row_base >> 16;
-        const uint32_t blk_kept_base = run_gt + min(run_eq, q);   // == gpos
-
-        uint32_t keep8[kVpl];
-#pragma unroll
-        for (int j = 0; j < kVpl; ++j) {
-            const uint32_t gt_before = run_gt + (excl[j] & 0xFFFFu);
-            const uint32_t eq_before = run_eq + (excl[j] >> 16);
-            uint32_t keep_eq = eq8[j];
-            if (keep_eq) {
-                const uint32_t room = (eq_before < q) ? (q - eq_before) : 0u;
-                if (room < (cnt[j] >> 16)) {
-                    uint32_t m = keep_eq;
-                    keep_eq = 0;
-                    for (uint32_t r = 0; r < room; ++r) {
-                        keep_eq |= m & (0u - m);
-                        m &= m - 1;
-                    }
-                }
-            }
-            keep8[j] = gt8[j] | keep_eq;
-            const uint32_t kept_before = gt_before + min(eq_before, q);
-            if constexpr (FULL) {   // vector blk*64 + j*32 + lane opens chunk blk*4 + j*2 + lane/16 when lane % 16 == 0
-                if ((lane & 15) == 0) offsets[blk * (kBlkElems / DROPIT_CHUNK) + j * 2 + (lane >> 4)] = kept_before;
+        uint32_t pos = run_gt + (excl & 0xFFFFu) + min(eq_before, q);   // retained elements before this lane's first
+        if ((lane & 7) == 0) {   // the lane opens a 128-element chunk
+            if constexpr (FULL) {
+                offsets[blk * (kBlkElems / DROPIT_CHUNK) + (lane >> 3)] = pos;
             } else {
-                const int64_t vi = blk * kBlkVecs + j * 32 + lane;
-                if ((lane & 15) == 0 && vi * 8 < n) offsets[(vi * 8) / DROPIT_CHUNK] = kept_before;
-            }
-            uint32_t pos = kept_before - blk_kept_base;
-            const uint32_t w[4] = {cur[j].x, cur[j].y, cur[j].z, cur[j].w};
-            [[maybe_unused]] const int32_t first_idx = (int32_t)(blk * kBlkElems) + (j * 32 + lane) * 8;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                if ((keep8[j] >> e) & 1u) {
-                    s_vals[pend + pos] = (uint16_t)((w[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu);
-                    if constexpr (INDEX32) s_idx[pend_i + pos] = first_idx + e;
-                    ++pos;
-                }
+                if (blk * kBlkElems + lane * 16 < n) offsets[blk * (kBlkElems / DROPIT_CHUNK) + (lane >> 3)] = pos;
             }
         }
         if constexpr (!INDEX32) {
-            // lanes sharing a 32-bit mask word OR their bytes, then lane i takes word i of the block
-            uint32_t word[kVpl];
-#pragma unroll
-            for (int j = 0; j < kVpl; ++j) {
-                uint32_t wv = keep8[j] << (8 * (lane & 3));
-                wv |= __shfl_xor_sync(kFullMask, wv, 1);
-                wv |= __shfl_xor_sync(kFullMask, wv, 2);
-                word[j] = wv;
-            }
-            uint32_t mine = 0;
-            const int src = (lane & 7) * 4;
-#pragma unroll
-            for (int j = 0; j < kVpl; ++j) {
-                const uint32_t got = __shfl_sync(kFullMask, word[j], src);
-                if ((lane >> 3) == j) mine = got;
-            }
-            const int64_t w0 = blk * (kBlkElems / 32);
+            uint32_t wv = keep << (16 * (lane & 1));
+            wv |= __shfl_xor_sync(kFullMask, wv, 1);
+            const int64_t wi = blk * (kBlkElems / 32) + (lane >> 1);
             if constexpr (FULL) {
-                if (lane < 8 * kVpl) mask[w0 + lane] = mine;
+                if (!(lane & 1)) mask[wi] = wv;
             } else {
-                if (lane < 8 * kVpl && w0 + lane < nwords) mask[w0 + lane] = mine;
+                if (!(lane & 1) && wi < nwords) mask[wi] = wv;
             }
         }
-        const uint32_t kept = (run_gt + blk_gt + min(run_eq + blk_eq, q)) - blk_kept_base;
-        run_gt += blk_gt;
-        run_eq += blk_eq;
-        __syncwarp();
-        flush_pieces<uint16_t, 8>(s_vals, values + (gpos - pend), kept, pend, foreign, lane);
-        if constexpr (INDEX32) flush_pieces<int32_t, 4>(s_idx, indices + (gpos - pend_i), kept, pend_i, foreign_i, lane);
-        gpos += kept;
+        {
+            // retained elements, lowest first: read from the ring, staged at their final position
+            [[maybe_unused]] const int32_t first_idx = (int32_t)(blk * kBlkElems) + lane * 16;
+            const uint32_t flip = swz << 4;   // element e of the lane sits at byte (2 * e) ^ flip of its 32
+            uint32_t m = keep;
+            while (m) {
+                const uint32_t e = (uint32_t)__ffs((int)m) - 1u;
+                m &= m - 1u;
+                uint16_t v;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(own + ((2u * e) ^ flip)) : "memory");
+                asm volatile("st.shared.u16 [%0], %1;" ::"r"(s_vals_addr + 2u * (pos & (kStageCap - 1))), "h"(v) : "memory");
+                if constexpr (INDEX32) indices[pos] = first_idx + (int32_t)e;
+                ++pos;
+            }
+        }
+        run_gt += tot & 0xFFFFu;
+        run_eq += tot >> 16;
+        gpos = run_gt + min(run_eq, q);
+        __syncwarp();   // staged values visible to the warp; every lane is done with the ring slot
+        if (gpos - head >= (uint32_t)kFlushVals) flush((gpos - head) / 8);
     };
     {
         int64_t blk = blk0;
         for (; blk < blk_full_end; ++blk) compact_block(blk, std::true_type{});
         for (; blk < blk1; ++blk) compact_block(blk, std::false_type{});
     }
-    // tails: own values still staged (less than one 16-byte piece); leading foreign slots are skipped
-    if (lane >= (int)foreign && lane < (int)pend) values[(gpos - pend) + lane] = s_vals[lane];
-    if constexpr (INDEX32) {
-        if (lane >= (int)foreign_i && lane < (int)pend_i) indices[(gpos - pend_i) + lane] = s_idx[lane];
-    }
+    // what is still staged: whole pieces, then the elements of the last, partial piece (the warp
+    // behind this one writes the rest of that piece)
+    flush((gpos - head) / 8);
+    if (lane >= (int)foreign && head + lane < gpos) values[head + lane] = s_vals[(head + lane) & (kStageCap - 1)];
     phase_stamp(st, 5);
 }
 
@@ -882,46 +945,25 @@ dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool inde
     const FusedPlan plan = make_fused_plan(n);
     if (workspace_bytes < plan.total_bytes) return DROPIT_ERR_WORKSPACE;
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
-    const size_t smem_hist = (size_t)kKeySpace * 4;   // sample kernel: one full key histogram
-    static_assert(kRingBytes >= (size_t)kKeySpace * 4, "the general path's histogram lives in the ring's memory");
-    const size_t smem_mask = kRingBytes + (size_t)kFusedWarps * kStageVals * 2;
-    const size_t smem_idx = smem_mask + (size_t)kFusedWarps * kStageIdx * 4;
+    static_assert(kRingBytes >= (size_t)kKeySpace * 4, "the sample's and the general path's histogram live in the ring's memory");
+    const size_t smem_mask = kRingBytes + kStageBytes + sizeof(FusedShared);
+    const size_t smem_idx = smem_mask;   // indices are written from registers, not staged
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(sample_band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_hist) != cudaSuccess ||
-            cudaFuncSetAttribute(fused_compress_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_mask) != cudaSuccess ||
+        if (cudaFuncSetAttribute(fused_compress_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_mask) != cudaSuccess ||
             cudaFuncSetAttribute(fused_compress_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_idx) != cudaSuccess)
             return DROPIT_ERR_CUDA;
         attr_set = true;
     }
-    {
-        cudaLaunchAttribute pdl[1];
-        pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        pdl[0].val.programmaticStreamSerializationAllowed = 1;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(1);
-        cfg.blockDim = dim3(kSampleThreads);
-        cfg.dynamicSmemBytes = smem_hist;
-        cfg.stream = stream;
-        cfg.attrs = pdl;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, sample_band_kernel, reinterpret_cast<const uint4*>(x), n, (unsigned long long)k, ws,
-                               plan.zero_bytes) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return DROPIT_ERR_CUDA;
-        }
-    }
-    dropit_status s = check_launch();
-    if (s != DROPIT_OK) return s;
-
     const uint4* xp = reinterpret_cast<const uint4*>(x);
     unsigned long long kk = (unsigned long long)k;
     int bpw = plan.blocks_per_warp;
+    uint32_t epoch = next_epoch();
     size_t h0 = plan.hist_off[0], h1 = plan.hist_off[1], ao = plan.agg_off, ro = plan.rows_off;
     uint16_t* vals = reinterpret_cast<uint16_t*>(values);
     uint32_t* maskp = index32 ? nullptr : reinterpret_cast<uint32_t*>(meta);
     int32_t* idxp = index32 ? reinterpret_cast<int32_t*>(meta) : nullptr;
-    void* args[] = {&xp, &n, &kk, &bpw, &ws, &h0, &h1, &ao, &ro, &vals, &maskp, &idxp, &offsets, &dev_status};
+    void* args[] = {&xp, &n, &kk, &bpw, &epoch, &ws, &h0, &h1, &ao, &ro, &vals, &maskp, &idxp, &offsets, &dev_status};
     const void* fn = index32 ? (const void*)fused_compress_kernel<true> : (const void*)fused_compress_kernel<false>;
     if (cudaLaunchCooperativeKernel(fn, dim3(plan.grid), dim3(kFusedThreads), args, index32 ? smem_idx : smem_mask,
                                     stream) != cudaSuccess) {
@@ -991,7 +1033,7 @@ extern "C" dropit_status dropit_compress_static(const void* x, int64_t n, double
     if (fused_compress_workspace_bytes(n) > kStaticScratchBytes) return DROPIT_ERR_WORKSPACE;
     unsigned char* scratch = static_scratch_address();
     if (!scratch) return DROPIT_ERR_CUDA;
-    // the sample kernel zeroes the part of the scratch that must start at zero on every call
+    // nothing in the scratch has to be cleared first (see the grid barrier); the kernel zeroes its own totals
     return fused_compress_bf16(x, n, k, format == DROPIT_FMT_INDEX32, values, meta, offsets, scratch,
                                kStaticScratchBytes, dev_status, stream);
 }
