@@ -5,7 +5,9 @@ the CUDA library.  torch supplies device memory and the current stream.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
+import functools
 from dataclasses import dataclass
 from typing import Optional, Tuple
 
@@ -49,11 +51,13 @@ def _check(code: int, where: str):
         raise DropITError(code, where)
 
 
+@functools.lru_cache(maxsize=4096)
 def dropit_keep_count(n: int, gamma: float) -> int:
     """k = n - ceil(gamma*n - 1e-6): retained elements at drop ratio gamma (Sec. 3.3, Sec. 4.1)."""
     return int(_lib.load().dropit_keep_count(int(n), float(gamma)))
 
 
+@functools.lru_cache(maxsize=4096)
 def dropit_cache_sizes(n: int, gamma: float, dtype: int, fmt: int) -> Tuple[int, int, int, int]:
     """(values_bytes, meta_bytes, offsets_bytes, workspace_bytes) for dropit_compress."""
     out = [ctypes.c_size_t(0) for _ in range(4)]
@@ -108,6 +112,13 @@ def _stream_ptr(device) -> ctypes.c_void_p:
     return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
 
 
+def _on_device(dev: torch.device):
+    """Make `dev` the current CUDA device for the call; free when it already is."""
+    if dev.index is None or dev.index == torch.cuda.current_device():
+        return contextlib.nullcontext()
+    return torch.cuda.device(dev)
+
+
 def _require_cuda(t: torch.Tensor, name: str):
     if not t.is_cuda:
         raise ValueError("%s must be a CUDA tensor (there is no CPU path)" % name)
@@ -132,7 +143,7 @@ def dropit_compress(x: torch.Tensor, gamma: float, fmt="bitmask", workspace: Opt
     offsets = torch.empty(ob // 4, dtype=torch.int32, device=dev)
     if workspace is None or workspace.numel() < wb:
         workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         code = lib.dropit_compress(_ptr(x), n, float(gamma), dt, fmt, _ptr(values), _ptr(meta), _ptr(offsets),
                                    _ptr(workspace), workspace.numel(), _ptr(_status_word(dev)), _stream_ptr(dev))
     _check(code, "dropit_compress")
@@ -144,13 +155,14 @@ def dropit_decompress(cache: DropITCache) -> torch.Tensor:
     lib = _lib.load()
     dev = cache.offsets.device if cache.offsets.numel() else cache.values.device
     out = torch.empty(cache.shape, dtype=cache.dtype, device=dev)
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         code = lib.dropit_decompress(_ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), cache.n, cache.k,
                                      _DTYPE_CODE[cache.dtype], cache.fmt, _ptr(out), _stream_ptr(dev))
     _check(code, "dropit_decompress")
     return out
 
 
+@functools.lru_cache(maxsize=4096)
 def dropit_weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int) -> int:
     out = ctypes.c_size_t(0)
     _check(_lib.load().dropit_weight_grad_workspace(M, Ca, Cz, dtype, fmt, ctypes.byref(out)),
@@ -182,7 +194,7 @@ def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch
     wb = dropit_weight_grad_workspace(M, Ca, Cz, dt, cache.fmt)
     if workspace is None or workspace.numel() < wb:
         workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         fn = lib.dropit_weight_grad_fused if fused else lib.dropit_weight_grad
         code = fn(_ptr(dy), _ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), M, Ca, Cz,
                                       cache.k, dt, cache.fmt, _ptr(out), int(bool(accumulate)), _ptr(workspace),
@@ -191,6 +203,7 @@ def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch
     return out
 
 
+@functools.lru_cache(maxsize=4096)
 def dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype: int, fmt: int) -> int:
     out = ctypes.c_size_t(0)
     _check(_lib.load().dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype, fmt,
@@ -218,7 +231,7 @@ def dropit_conv_weight_grad(dy: torch.Tensor, cache: DropITCache, kernel_size: T
     wb = dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dt, cache.fmt)
     if workspace is None or workspace.numel() < wb:
         workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         code = lib.dropit_conv_weight_grad(_ptr(dy), _ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), B, Ca,
                                            H, W, Cz, R, S, stride, pad, dilation, cache.k, dt, cache.fmt, _ptr(out),
                                            int(bool(accumulate)), _ptr(workspace), workspace.numel(),

@@ -46,13 +46,16 @@ constexpr int kSampleVecs = 2048;                              // 16384 sampled 
 constexpr int64_t kSampleMinElems = 1 << 19;                   // below this the band is the full key range
 constexpr int kBarrierSpinLimit = 1 << 22;
 constexpr uint32_t kHiBits = 0x80008000u;
-constexpr int kRingDepth = 4;                                  // blocks of a warp's run in flight (cp.async ring)
-constexpr int kRingSlotBytes = kBlkVecs * 16;                  // one block
-constexpr size_t kRingBytes = (size_t)kFusedWarps * kRingDepth * kRingSlotBytes;   // 128 KB
-constexpr int kStageCap = 1024;                                // per-warp circular staging of retained values (power of two)
-constexpr int kFlushVals = 256;                                // staged values that trigger a flush: one 16-byte piece per lane
-static_assert(kFlushVals + kBlkElems + 8 <= kStageCap, "a block must fit behind what a flush leaves");
-constexpr size_t kStageBytes = (size_t)kFusedWarps * kStageCap * 2;   // 64 KB
+// The streaming passes work on super-blocks of two blocks (1024 elements): a lane owns 32 CONSECUTIVE
+// elements, i.e. one mask word.  Each warp has a ring of two super-block slots fed by cp.async.
+constexpr int kSbVecs = 2 * kBlkVecs;                          // 128 vectors
+constexpr int kSbElems = 2 * kBlkElems;                        // 1024 bf16
+constexpr int kSbBytes = kSbVecs * 16;                         // 2 KB
+constexpr int kSbChunks = kSbElems / DROPIT_CHUNK;             // 8 seek-table entries
+constexpr int kRingSlots = 2;
+constexpr size_t kRingBytes = (size_t)kFusedWarps * kRingSlots * kSbBytes;   // 128 KB
+constexpr int kStageVals = kSbElems + 8;                       // per-warp staging: a super-block's retained values behind < 8 carried ones
+constexpr size_t kStageBytes = (size_t)kFusedWarps * kStageVals * 2;   // 64.5 KB
 static_assert(kStageBytes >= (size_t)kKeySpace * 2, "the sample's 16-bit histogram lives in the staging area");
 
 struct FusedState {
@@ -81,6 +84,7 @@ static FusedPlan make_fused_plan(int64_t n) {
     p.grid = g;
     p.blocks_per_warp = (int)((p.blocks_total + (int64_t)g * kFusedWarps - 1) / ((int64_t)g * kFusedWarps));
     if (p.blocks_per_warp < 1) p.blocks_per_warp = 1;
+    p.blocks_per_warp = (p.blocks_per_warp + 1) & ~1;          // a run is a whole number of super-blocks
     p.hist_off[0] = kStateBytes;
     p.hist_off[1] = p.hist_off[0] + (size_t)kKeySpace * 4;
     p.agg_off = p.hist_off[1] + (size_t)kKeySpace * 4;
@@ -183,10 +187,6 @@ __device__ __forceinline__ void phase_stamp(FusedState*, int) {}
 // same band without any exchange.  `bins`: kKeySpace counters in shared memory; band[0..1] = lo, hi.
 // Ends with a block-wide barrier.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t sample_count(const uint32_t* bins, uint32_t key) {
-    return (bins[key >> 1] >> ((key & 1u) * 16)) & 0xFFFFu;
-}
-
 template <typename AfterLoads>
 __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t n, unsigned long long k, uint32_t* bins,
                                             uint32_t* s_warp, uint32_t* band, FusedState* st, AfterLoads after_loads) {
@@ -230,13 +230,20 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
         const float r_hi = ks - margin, r_lo = ks + margin;
         constexpr int PER = kKeySpace / kFusedThreads;   // keys per thread, descending: kKeySpace-1 - (t*PER + r)
         const int t = threadIdx.x;
-        const uint32_t* mine = bins + (kKeySpace / 2 - (t + 1) * (PER / 2));   // the thread's PER/2 words
+        static_assert(PER == 32, "the walk below assumes 16 words per thread");
+        // the thread's 16 words, kept in registers for the walk below
+        uint32_t cw[PER / 2];
+        {
+            const uint4* mine = reinterpret_cast<const uint4*>(bins + (kKeySpace / 2 - (t + 1) * (PER / 2)));
+#pragma unroll
+            for (int j = 0; j < PER / 8; ++j) {
+                const uint4 v = mine[j];
+                cw[4 * j] = v.x; cw[4 * j + 1] = v.y; cw[4 * j + 2] = v.z; cw[4 * j + 3] = v.w;
+            }
+        }
         uint32_t sum = 0;
 #pragma unroll
-        for (int r = 0; r < PER / 2; ++r) {
-            const uint32_t w = mine[(r + t) & (PER / 2 - 1)];   // rotated start: fewer bank conflicts
-            sum += (w & 0xFFFFu) + (w >> 16);
-        }
+        for (int r = 0; r < PER / 2; ++r) sum += (cw[r] & 0xFFFFu) + (cw[r] >> 16);
         uint32_t total;
         const uint32_t excl = block_exclusive_scan(sum, s_warp, &total);
         phase_stamp(st, 10);
@@ -244,9 +251,12 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
         if ((r_hi >= 1.0f && (float)excl < r_hi && r_hi <= (float)(excl + sum)) ||
             (r_lo <= S && (float)excl < r_lo && r_lo <= (float)(excl + sum))) {
             uint32_t cum = excl;
+#pragma unroll
             for (int r = 0; r < PER; ++r) {
+                // key = kKeySpace-1 - (t*PER + r) lives in word 15 - r/2 of the thread, upper half when r is even
                 const uint32_t key = kKeySpace - 1 - (t * PER + r);
-                const uint32_t hh = sample_count(bins, key);
+                const uint32_t cwr = cw[PER / 2 - 1 - r / 2];
+                const uint32_t hh = (r & 1) ? (cwr & 0xFFFFu) : (cwr >> 16);
                 if (hh) {
                     if (r_hi >= 1.0f && (float)cum < r_hi && r_hi <= (float)(cum + hh)) band[1] = key;
                     if (r_lo <= S && (float)cum < r_lo && r_lo <= (float)(cum + hh)) band[0] = key;
@@ -282,7 +292,8 @@ struct FusedShared {
 // in this call.  Every wait is bounded: returns false when one runs out.
 __device__ __forceinline__ void barrier_open(unsigned long long* word, uint32_t epoch) {
     if (blockIdx.x == 0 && threadIdx.x == 0) {
-        asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(word), "l"((unsigned long long)epoch << 32) : "memory");
+        // relaxed: nothing is published with it, and the other CTAs look for it microseconds later
+        asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(word), "l"((unsigned long long)epoch << 32) : "memory");
     }
 }
 __device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t epoch, uint32_t target, int* s_ok) {
@@ -359,15 +370,16 @@ __device__ __forceinline__ void load_block(const uint4* x, int64_t blk, int lane
     }
 }
 
-// The warp's blocks are streamed through a per-warp ring in shared memory fed by cp.async, several
-// blocks ahead, so that enough bytes are in flight per SM without holding them in registers.  Each
-// lane copies and later reads only its own 16-byte vectors, so a cp.async.wait_group is all the
-// synchronisation the ring needs.  `lane_slot` = shared address of the lane's first vector in the slot.
-__device__ __forceinline__ void ring_issue(uint32_t lane_slot, const uint4* x, int64_t blk, int lane, int64_t nvec_full,
-                                           int64_t n) {
+// The warp's super-blocks are streamed through a per-warp ring in shared memory fed by cp.async, one
+// super-block ahead, so that enough bytes are in flight per SM without holding them in registers.
+// The copies are coalesced (lane copies vectors lane, lane+32, lane+64, lane+96 of the super-block);
+// a lane then reads the 64 bytes at 64*lane, which other lanes copied, so a __syncwarp follows the wait.
+// `lane_slot` = shared address of vector `lane` in the slot.
+__device__ __forceinline__ void sb_issue_edge(uint32_t lane_slot, const uint4* x, int64_t sb, int lane, int64_t nvec_full,
+                                              int64_t n) {
 #pragma unroll
-    for (int j = 0; j < kVpl; ++j) {
-        const int64_t vi = blk * kBlkVecs + j * 32 + lane;
+    for (int j = 0; j < kSbVecs / 32; ++j) {
+        const int64_t vi = sb * kSbVecs + j * 32 + lane;
         const uint32_t dst = lane_slot + j * 512;
         if (vi == nvec_full && (n & 7) != 0) {   // ragged last vector of the tensor: assembled by hand
             int nv;
@@ -383,25 +395,41 @@ __device__ __forceinline__ void ring_issue(uint32_t lane_slot, const uint4* x, i
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
-// The same for a block whose vectors are all whole: `src` = the lane's first vector of the block.
-__device__ __forceinline__ void ring_issue_full(uint32_t lane_slot, const uint4* src) {
+// The same for a super-block whose vectors are all whole: `src` = vector `lane` of the super-block.
+__device__ __forceinline__ void sb_issue_full(uint32_t lane_slot, const uint4* src) {
 #pragma unroll
-    for (int j = 0; j < kVpl; ++j)
+    for (int j = 0; j < kSbVecs / 32; ++j)
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(lane_slot + j * 512), "l"(src + j * 32) : "memory");
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
-__device__ __forceinline__ void ring_read(uint32_t lane_slot, uint4 (&v)[kVpl]) {
+// The lane's 32 elements (16 words) of a slot; `own` = shared address of the slot + 64 * lane.
+__device__ __forceinline__ void sb_read(uint32_t own, uint32_t (&w)[16]) {
 #pragma unroll
-    for (int j = 0; j < kVpl; ++j)
+    for (int j = 0; j < 4; ++j)
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(v[j].x), "=r"(v[j].y), "=r"(v[j].z), "=r"(v[j].w)
-                     : "r"(lane_slot + j * 512)
+                     : "=r"(w[4 * j]), "=r"(w[4 * j + 1]), "=r"(w[4 * j + 2]), "=r"(w[4 * j + 3])
+                     : "r"(own + j * 16)
                      : "memory");
 }
-// The block issued kRingDepth-1 commits ago has landed.
-__device__ __forceinline__ void ring_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kRingDepth - 1) : "memory"); }
+// All but the most recently committed super-block have landed.
+__device__ __forceinline__ void sb_wait() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ int valid_elems(int64_t vi, int64_t nvec_full, int64_t n) {
     return vi < nvec_full ? 8 : (vi == nvec_full ? (int)(n & 7) : 0);
+}
+__device__ __forceinline__ uint32_t top_bit(uint32_t m) {   // index of the highest set bit (m != 0)
+    uint32_t e;
+    asm("bfind.u32 %0, %1;" : "=r"(e) : "r"(m));
+    return e;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+// Mask of the lane's elements that exist: the lane owns [first, first + 32) of a tensor of n elements.
+__device__ __forceinline__ uint32_t valid_mask32(int64_t first, int64_t n) {
+    const int64_t left = n - first;
+    return left >= 32 ? 0xFFFFFFFFu : (left > 0 ? (1u << (int)left) - 1u : 0u);
 }
 
 template <bool INDEX32>
@@ -416,24 +444,29 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     extern __shared__ __align__(16) unsigned char fsm[];
     uint32_t* bins = reinterpret_cast<uint32_t*>(fsm);
     uint32_t* sample_bins = reinterpret_cast<uint32_t*>(fsm + kRingBytes);
-    uint16_t* s_vals_all = reinterpret_cast<uint16_t*>(fsm + kRingBytes);
+    uint16_t* s_vals_all = reinterpret_cast<uint16_t*>(fsm + kRingBytes);   // phase 3: per-warp staging
     FusedShared& sh = *reinterpret_cast<FusedShared*>(fsm + kRingBytes + kStageBytes);
 
     FusedState* st = reinterpret_cast<FusedState*>(ws);
     unsigned long long* agg = reinterpret_cast<unsigned long long*>(ws + agg_off);
     uint32_t* rows = reinterpret_cast<uint32_t*>(ws + rows_off);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t ring_lane = ptx_smem(fsm) + (warp * kRingDepth) * kRingSlotBytes + lane * 16;
+    const uint32_t ring_warp = ptx_smem(fsm) + warp * (kRingSlots * kSbBytes);
+    const uint32_t ring_copy = ring_warp + lane * 16;   // where the lane's copies of a slot start
+    const uint32_t ring_own = ring_warp + lane * 64;    // the lane's 32 elements of a slot
     const int64_t nvec_full = n / 8;
     const int64_t blocks_total = (n + kBlkElems - 1) / kBlkElems;
-    const int64_t blk0 = ((int64_t)blockIdx.x * kFusedWarps + warp) * blocks_per_warp;
+    const int64_t blk0 = ((int64_t)blockIdx.x * kFusedWarps + warp) * blocks_per_warp;   // even
     int64_t blk1 = blk0 + blocks_per_warp;
     if (blk1 > blocks_total) blk1 = blocks_total;
-    // blocks below this index consist of whole vectors only: they take the paths without bounds arithmetic
-    const int64_t blk_full_end = (nvec_full / kBlkVecs < blk1) ? nvec_full / kBlkVecs : blk1;
-    auto issue_block = [&](int64_t b, uint32_t dst) {
-        if (b < blk_full_end) ring_issue_full(dst, x + b * kBlkVecs + lane);
-        else if (b < blk1) ring_issue(dst, x, b, lane, nvec_full, n);
+    // the same run in super-blocks; those below sb_full_end consist of whole vectors only and take the
+    // paths without bounds arithmetic
+    const int64_t sb0 = blk0 / 2, sb1 = (blk1 + 1) / 2;
+    const int64_t sb_full_end = (nvec_full / kSbVecs < sb1) ? nvec_full / kSbVecs : sb1;
+    auto issue_sb = [&](int64_t sb, int slot) {
+        const uint32_t dst = ring_copy + slot * kSbBytes;
+        if (sb < sb_full_end) sb_issue_full(dst, x + sb * kSbVecs + lane);
+        else if (sb < sb1) sb_issue_edge(dst, x, sb, lane, nvec_full, n);
         else asm volatile("cp.async.commit_group;" ::: "memory");
     };
     uint32_t barrier_target = 0;
@@ -447,10 +480,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     barrier_open(&st->barrier, epoch);
     // the first blocks of the run are requested right behind the sample loads, whose processing hides their latency
     bool prefetched = true;
-    sample_band(x, n, k, sample_bins, sh.warp, sh.band, st, [&] {
-#pragma unroll
-        for (int d = 0; d < kRingDepth - 1; ++d) issue_block(blk0 + d, ring_lane + d * kRingSlotBytes);
-    });
+    sample_band(x, n, k, sample_bins, sh.warp, sh.band, st, [&] { issue_sb(sb0, 0); });
     uint32_t lo = sh.band[0], hi = sh.band[1];
     uint32_t T = 0, q = 0;
     uint32_t run_gt = 0, run_eq = 0;   // this warp's exclusive prefix (absolute)
@@ -507,28 +537,46 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             }
         };
         if (narrow) {
-            // stream the run through the ring, kRingDepth-1 blocks ahead
-            if (!prefetched) {
+            // stream the run through the ring, one super-block ahead
+            if (!prefetched) issue_sb(sb0, 0);
+            int slot = 0;
+            auto count_sb = [&](int64_t sb, auto full_tag) {
+                constexpr bool FULL = decltype(full_tag)::value;
+                issue_sb(sb + 1, slot ^ 1);
+                sb_wait();
+                __syncwarp();   // the lane reads vectors that other lanes copied
+                const uint32_t own = ring_own + slot * kSbBytes;
+                uint32_t w[16];
+                sb_read(own, w);
+                uint32_t hi_flags = 0, pending = 0;
 #pragma unroll
-                for (int d = 0; d < kRingDepth - 1; ++d) issue_block(blk0 + d, ring_lane + d * kRingSlotBytes);
-            }
-            int slot = 0, slot_ahead = kRingDepth - 1;
-            for (int64_t blk = blk0; blk < blk1; ++blk) {
-                issue_block(blk + kRingDepth - 1, ring_lane + slot_ahead * kRingSlotBytes);
-                ring_wait();
-                uint4 va[kVpl];
-                ring_read(ring_lane + slot * kRingSlotBytes, va);
-                if (blk < blk_full_end) {
+                for (int g = 0; g < 4; ++g) {   // four words = eight elements at a time
+                    uint32_t a[4], b[4];
 #pragma unroll
-                    for (int j = 0; j < kVpl; ++j) count_vec(va[j], 8);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < kVpl; ++j)
-                        count_vec(va[j], valid_elems(blk * kBlkVecs + j * 32 + lane, nvec_full, n));
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t m = w[4 * g + i] & 0x7FFF7FFFu;
+                        a[i] = m + c_hi;                   // bit 15 of a half: key > hi
+                        b[i] = (m + c_lo) & ~a[i];         // bit 15 of a half: lo <= key <= hi
+                    }
+                    // above the band only the count matters: the flag bytes of all 16 words share one word
+                    hi_flags |= ((__byte_perm(a[0], a[1], 0x7531) & 0x80808080u) >> (2 * g)) |
+                                ((__byte_perm(a[2], a[3], 0x7531) & 0x80808080u) >> (2 * g + 1));
+                    pending |= flags8(b[0], b[1], b[2], b[3]) << (8 * g);
                 }
-                slot = (slot + 1 == kRingDepth) ? 0 : slot + 1;
-                slot_ahead = (slot_ahead + 1 == kRingDepth) ? 0 : slot_ahead + 1;
-            }
+                cnt_hi += __popc(hi_flags);
+                if constexpr (!FULL) pending &= valid_mask32(sb * kSbElems + lane * 32, n);   // zero padding is no data
+                while (pending) {   // a few percent of the elements: the band histogram (their order is irrelevant)
+                    const uint32_t e = top_bit(pending);
+                    pending ^= 1u << e;
+                    const uint32_t d = (lds_u16(own + 2u * e) & 0x7FFFu) - lo;
+                    if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
+                }
+                __syncwarp();   // every lane is done with the slot before it is refilled
+                slot ^= 1;
+            };
+            int64_t sb = sb0;
+            for (; sb < sb_full_end; ++sb) count_sb(sb, std::true_type{});
+            for (; sb < sb1; ++sb) count_sb(sb, std::false_type{});
             asm volatile("cp.async.wait_all;" ::: "memory");
         } else {
             int64_t blk = blk0;
@@ -786,82 +834,48 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     __syncthreads();   // shared histograms are dead from here on; phase 3 reuses the memory
     phase_stamp(st, 3);
 
-    // ---------------- phase 3: ordered compaction, one warp per run of blocks ----------------
-    // A lane owns 16 CONSECUTIVE elements of a block (vectors 2*lane and 2*lane+1), i.e. half a mask
-    // word, so a block costs one warp scan and one shuffle for the mask.  The copies into the ring
-    // stay coalesced (lane copies vectors lane and lane+32); vector v sits at 16-byte position
-    // v ^ ((v >> 3) & 1) of its slot so that neither side has bank conflicts.  Retained values go to
-    // a per-warp circular buffer indexed by their final position in `values` (mod kStageCap) and
-    // leave for global memory as one aligned 16-byte piece per lane once kFlushVals are staged.
+    // ---------------- phase 3: ordered compaction, one warp per run of super-blocks ----------------
+    // A lane owns 32 consecutive elements = one mask word, so a super-block costs one warp scan and the
+    // mask needs no exchange.  Retained values are staged per warp at (final position - head) and leave
+    // for global memory in aligned 16-byte pieces after every super-block; the < 8 that remain are
+    // carried to the front of the buffer.
     ptx::launch_dependents();   // a programmatically launched kernel behind this one may be brought up
     const int64_t nwords = (n + 31) / 32;
-    uint16_t* s_vals = s_vals_all + (size_t)warp * kStageCap;
+    uint16_t* s_vals = s_vals_all + (size_t)warp * kStageVals;
     const uint32_t s_vals_addr = ptx_smem(s_vals);
     const uint32_t c_gt = ge_const(T + 1), c_ge = ge_const(T);
-    const uint32_t ring_warp = ptx_smem(fsm) + (warp * kRingDepth) * kRingSlotBytes;
-    const uint32_t ring_copy = ring_warp + ((lane ^ ((lane >> 3) & 1)) * 16);   // where vector `lane` of a slot goes
-    const uint32_t swz = (lane >> 2) & 1;                                        // swizzle bit of vectors 2*lane, 2*lane+1
-    const uint32_t ring_own = ring_warp + lane * 32;                             // the lane's 32 bytes of a slot
-    auto issue3 = [&](int64_t b, uint32_t dst) {
-        if (b < blk_full_end) ring_issue_full(dst, x + b * kBlkVecs + lane);
-        else if (b < blk1) ring_issue(dst, x, b, lane, nvec_full, n);
-        else asm volatile("cp.async.commit_group;" ::: "memory");
-    };
-    uint32_t gpos = run_gt + min(run_eq, q);   // retained elements before this warp's next block
+    uint32_t gpos = run_gt + min(run_eq, q);   // retained elements before this warp's next super-block
     uint32_t head = gpos & ~7u;                // first position not yet written to `values` (16-byte aligned)
     uint32_t foreign = gpos & 7u;              // leading slots of the first piece that belong to the previous warp
-    // Write staged positions [head, head + 8 * pieces): piece c by lane c % 32.
-    auto flush = [&](uint32_t pieces) {
-        for (uint32_t c = lane; c < pieces; c += 32) {
-            const uint32_t p = head + c * 8;
-            if (c == 0 && foreign) {
-                for (uint32_t e = foreign; e < 8; ++e) values[p + e] = s_vals[(p + e) & (kStageCap - 1)];
-            } else {
-                *reinterpret_cast<uint4*>(values + p) = *reinterpret_cast<const uint4*>(s_vals + (p & (kStageCap - 1)));
-            }
-        }
-        if (pieces) foreign = 0;
-        head += pieces * 8;
-        __syncwarp();   // the slots may be staged again only after every lane has read its piece
-    };
-#pragma unroll
-    for (int d = 0; d < kRingDepth - 1; ++d) issue3(blk0 + d, ring_copy + d * kRingSlotBytes);
-    int slot = 0, slot_ahead = kRingDepth - 1;
-    // One block of the run.  FULL: every vector of the block is whole, so the bounds arithmetic folds away.
-    auto compact_block = [&](int64_t blk, auto full_tag) {
+    issue_sb(sb0, 0);
+    int slot = 0;
+    auto compact_sb = [&](int64_t sb, auto full_tag) {
         constexpr bool FULL = decltype(full_tag)::value;
-        issue3(blk + kRingDepth - 1, ring_copy + slot_ahead * kRingSlotBytes);
-        ring_wait();
+        issue_sb(sb + 1, slot ^ 1);
+        sb_wait();
         __syncwarp();   // the lane reads vectors that other lanes copied
-        const uint32_t own = ring_own + slot * kRingSlotBytes;
-        uint32_t w[8];
-        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(own + swz * 16) : "memory");
-        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(own + (swz ^ 1u) * 16) : "memory");
-        slot = (slot + 1 == kRingDepth) ? 0 : slot + 1;
-        slot_ahead = (slot_ahead + 1 == kRingDepth) ? 0 : slot_ahead + 1;
-        uint32_t a[8], eany = 0;
+        const uint32_t own = ring_own + slot * kSbBytes;
+        uint32_t g32 = 0, ge32 = 0;
+        {
+            uint32_t w[16];
+            sb_read(own, w);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t m = w[i] & 0x7FFF7FFFu;
-            a[i] = m + c_gt;                        // bit 15 of a half: key > T
-            eany |= (m + c_ge) & ~a[i];             // bit 15 of a half: key == T
-        }
-        const uint32_t g16 = flags8(a[0], a[1], a[2], a[3]) | (flags8(a[4], a[5], a[6], a[7]) << 8);
-        uint32_t e16 = 0;
-        if (eany & kHiBits) {
-            uint32_t eb[8];
+            for (int g = 0; g < 4; ++g) {
+                uint32_t a[4], b[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) eb[i] = ((w[i] & 0x7FFF7FFFu) + c_ge) & ~a[i];
-            e16 = flags8(eb[0], eb[1], eb[2], eb[3]) | (flags8(eb[4], eb[5], eb[6], eb[7]) << 8);
-            if constexpr (!FULL) {   // zero padding past the end must not tie with T = 0
-                const int64_t left = n - (blk * kBlkElems + lane * 16);
-                e16 &= left >= 16 ? 0xFFFFu : (left > 0 ? (1u << (int)left) - 1u : 0u);
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t m = w[4 * g + i] & 0x7FFF7FFFu;
+                    a[i] = m + c_gt;                       // bit 15 of a half: key > T
+                    b[i] = m + c_ge;                       // bit 15 of a half: key >= T
+                }
+                g32 |= flags8(a[0], a[1], a[2], a[3]) << (8 * g);
+                ge32 |= flags8(b[0], b[1], b[2], b[3]) << (8 * g);
             }
         }
-        const uint32_t cnt = __popc(g16) | (__popc(e16) << 16);
-        // packed (gt | eq << 16) prefix over the lanes = over the block's elements
+        uint32_t e32 = ge32 & ~g32;   // key == T
+        if constexpr (!FULL) e32 &= valid_mask32(sb * kSbElems + lane * 32, n);   // zero padding must not tie with T = 0
+        const uint32_t cnt = __popc(g32) | (__popc(e32) << 16);
+        // packed (gt | eq << 16) prefix over the lanes = over the super-block's elements
         uint32_t inc = cnt;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -871,12 +885,12 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         const uint32_t tot = __shfl_sync(kFullMask, inc, 31);
         const uint32_t excl = inc - cnt;
         const uint32_t eq_before = run_eq + (excl >> 16);
-        uint32_t keep = g16;
-        if (e16) {
+        uint32_t keep = g32;
+        if (e32) {
             const uint32_t room = (eq_before < q) ? (q - eq_before) : 0u;
-            uint32_t ke = e16;
+            uint32_t ke = e32;
             if (room < (cnt >> 16)) {   // the quota ends inside this lane's ties: the first `room` of them stay
-                uint32_t m = e16;
+                uint32_t m = e32;
                 ke = 0;
                 for (uint32_t r = 0; r < room; ++r) {
                     ke |= m & (0u - m);
@@ -885,54 +899,69 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             }
             keep |= ke;
         }
-        uint32_t pos = run_gt + (excl & 0xFFFFu) + min(eq_before, q);   // retained elements before this lane's first
-        if ((lane & 7) == 0) {   // the lane opens a 128-element chunk
+        const uint32_t pos = run_gt + (excl & 0xFFFFu) + min(eq_before, q);   // retained elements before this lane's first
+        if ((lane & 3) == 0) {   // the lane opens a 128-element chunk
             if constexpr (FULL) {
-                offsets[blk * (kBlkElems / DROPIT_CHUNK) + (lane >> 3)] = pos;
+                offsets[sb * kSbChunks + (lane >> 2)] = pos;
             } else {
-                if (blk * kBlkElems + lane * 16 < n) offsets[blk * (kBlkElems / DROPIT_CHUNK) + (lane >> 3)] = pos;
+                if (sb * kSbElems + lane * 32 < n) offsets[sb * kSbChunks + (lane >> 2)] = pos;
             }
         }
         if constexpr (!INDEX32) {
-            uint32_t wv = keep << (16 * (lane & 1));
-            wv |= __shfl_xor_sync(kFullMask, wv, 1);
-            const int64_t wi = blk * (kBlkElems / 32) + (lane >> 1);
+            const int64_t wi = sb * (kSbElems / 32) + lane;
             if constexpr (FULL) {
-                if (!(lane & 1)) mask[wi] = wv;
+                mask[wi] = keep;
             } else {
-                if (!(lane & 1) && wi < nwords) mask[wi] = wv;
+                if (wi < nwords) mask[wi] = keep;
             }
         }
         {
-            // retained elements, lowest first: read from the ring, staged at their final position
-            [[maybe_unused]] const int32_t first_idx = (int32_t)(blk * kBlkElems) + lane * 16;
-            const uint32_t flip = swz << 4;   // element e of the lane sits at byte (2 * e) ^ flip of its 32
+            // the lane's retained elements, highest first: read from the ring, staged at their final position
+            [[maybe_unused]] const int32_t first_idx = (int32_t)(sb * kSbElems) + lane * 32;
             uint32_t m = keep;
+            uint32_t p_abs = pos + __popc(keep);
             while (m) {
-                const uint32_t e = (uint32_t)__ffs((int)m) - 1u;
-                m &= m - 1u;
-                uint16_t v;
-                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(own + ((2u * e) ^ flip)) : "memory");
-                asm volatile("st.shared.u16 [%0], %1;" ::"r"(s_vals_addr + 2u * (pos & (kStageCap - 1))), "h"(v) : "memory");
-                if constexpr (INDEX32) indices[pos] = first_idx + (int32_t)e;
-                ++pos;
+                const uint32_t e = top_bit(m);
+                m ^= 1u << e;
+                --p_abs;
+                const uint32_t v = lds_u16(own + 2u * e);
+                asm volatile("st.shared.u16 [%0], %1;" ::"r"(s_vals_addr + 2u * (p_abs - head)), "r"(v) : "memory");
+                if constexpr (INDEX32) indices[p_abs] = first_idx + (int32_t)e;
             }
         }
         run_gt += tot & 0xFFFFu;
         run_eq += tot >> 16;
         gpos = run_gt + min(run_eq, q);
         __syncwarp();   // staged values visible to the warp; every lane is done with the ring slot
-        if (gpos - head >= (uint32_t)kFlushVals) flush((gpos - head) / 8);
+        slot ^= 1;
+        // write the whole 16-byte pieces, carry the rest to the front
+        const uint32_t staged = gpos - head;
+        const uint32_t pieces = staged / 8;
+        if (pieces) {
+            for (uint32_t c = lane; c < pieces; c += 32) {
+                if (c == 0 && foreign) {
+                    for (uint32_t e = foreign; e < 8; ++e) values[head + e] = s_vals[e];
+                } else {
+                    *reinterpret_cast<uint4*>(values + head + c * 8) = *reinterpret_cast<const uint4*>(s_vals + c * 8);
+                }
+            }
+            foreign = 0;
+            const uint32_t rem = staged - pieces * 8;
+            uint16_t carry = 0;
+            if (lane < (int)rem) carry = s_vals[pieces * 8 + lane];
+            __syncwarp();
+            if (lane < (int)rem) s_vals[lane] = carry;
+            head += pieces * 8;
+            __syncwarp();
+        }
     };
     {
-        int64_t blk = blk0;
-        for (; blk < blk_full_end; ++blk) compact_block(blk, std::true_type{});
-        for (; blk < blk1; ++blk) compact_block(blk, std::false_type{});
+        int64_t sb = sb0;
+        for (; sb < sb_full_end; ++sb) compact_sb(sb, std::true_type{});
+        for (; sb < sb1; ++sb) compact_sb(sb, std::false_type{});
     }
-    // what is still staged: whole pieces, then the elements of the last, partial piece (the warp
-    // behind this one writes the rest of that piece)
-    flush((gpos - head) / 8);
-    if (lane >= (int)foreign && head + lane < gpos) values[head + lane] = s_vals[(head + lane) & (kStageCap - 1)];
+    // the elements of the last, partial piece (the warp behind this one writes the rest of that piece)
+    if (lane >= (int)foreign && head + lane < gpos) values[head + lane] = s_vals[lane];
     phase_stamp(st, 5);
 }
 
