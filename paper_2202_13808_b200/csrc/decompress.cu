@@ -7,48 +7,89 @@ namespace dropit {
 unsigned long long g_launch_count = 0;
 
 // A warp inflates 1024 consecutive elements (32 mask words, 8 chunks) per step: lane l owns word l.
-// Its first retained element sits at the chunk's table entry plus the population of the chunk's
-// earlier words.  The lane drops its retained values into a zeroed shared-memory image of the 1024
-// elements (work proportional to the number of retained values, not to the dense size), and the warp
-// then streams the image out as 512-byte store instructions.
-constexpr int kDecompWarps = 8;
+// The retained values of a step are one contiguous piece of `values` (from the seek-table entry of the
+// step's first chunk to that of the next step), which the warp fetches with coalesced 16-byte loads into
+// shared memory.  Each lane then drops its values (they start at the chunk's table entry plus the
+// population of the chunk's earlier words) into a zeroed shared-memory image of the 1024 elements -
+// work proportional to the number of retained values, not to the dense size - and the warp streams the
+// image out as 512-byte store instructions.  The grid is persistent; the mask word and the table
+// entries of a warp's next step are requested before the current step is processed, so a step waits
+// for one round trip to memory (its values), not three.
+template <typename Tr> struct DecompWarps { static constexpr int value = Tr::kElemBytes == 2 ? 8 : 4; };   // 36 KB of shared memory per CTA either way
+constexpr int kDecompCtasPerSm = 6;
 
 template <typename Tr>
-__global__ void __launch_bounds__(32 * kDecompWarps)
+__global__ void __launch_bounds__(32 * DecompWarps<Tr>::value)
 decompress_bitmask_kernel(const typename Tr::elem_t* __restrict__ values, const uint32_t* __restrict__ mask,
-                          const uint32_t* __restrict__ offsets, int64_t n, typename Tr::elem_t* __restrict__ out) {
+                          const uint32_t* __restrict__ offsets, int64_t n, int64_t k,
+                          typename Tr::elem_t* __restrict__ out) {
     using elem_t = typename Tr::elem_t;
+    constexpr int kDecompWarps = DecompWarps<Tr>::value;
     constexpr int G = Tr::kVecElems;                 // elements per 16-byte vector
     constexpr int kPitch = 32 + G;                   // image row = one mask word; one spare vector spreads the banks
     constexpr int kVecPerRow = 32 / G;
+    constexpr int kSegElems = 1024 + G;              // a step's values, fetched from a 16-byte boundary
     __shared__ __align__(16) elem_t image[kDecompWarps][32 * kPitch];
+    __shared__ __align__(16) elem_t segment[kDecompWarps][kSegElems];
     ptx::grid_dependency_wait();   // launched programmatically: the cache may come from the kernel before this one
     ptx::launch_dependents();      // a weight-gradient kernel behind this one may set itself up meanwhile
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     elem_t* img = image[warp];
+    elem_t* seg = segment[warp];
     const int64_t nwords = (n + 31) / 32;
+    const int64_t nchunks = (n + DROPIT_CHUNK - 1) / DROPIT_CHUNK;
     const int64_t ntiles = (nwords + 31) / 32;
-    for (int64_t t = (int64_t)blockIdx.x * kDecompWarps + warp; t < ntiles; t += (int64_t)gridDim.x * kDecompWarps) {
+    const int64_t stride = (int64_t)gridDim.x * kDecompWarps;
+    // what a step needs before its values: the lane's mask word, and (lanes 0..8) the table entries of the
+    // step's eight chunks and of the chunk behind them (k past the end of the table)
+    auto fetch_word = [&](int64_t t) -> uint32_t {
         const int64_t w = t * 32 + lane;
-        uint32_t word = (w < nwords) ? __ldg(mask + w) : 0u;
-        const int64_t e_word = w * 32;
+        return (t < ntiles && w < nwords) ? __ldg(mask + w) : 0u;
+    };
+    auto fetch_entry = [&](int64_t t) -> uint32_t {
+        const int64_t c = t * 8 + lane;
+        if (t >= ntiles || lane > 8) return 0u;
+        return c < nchunks ? __ldg(offsets + c) : (uint32_t)k;
+    };
+    int64_t t = (int64_t)blockIdx.x * kDecompWarps + warp;
+    uint32_t word_next = fetch_word(t), entry_next = fetch_entry(t);
+    for (; t < ntiles; t += stride) {
+        uint32_t word = word_next;
+        const uint32_t entry = entry_next;
+        word_next = fetch_word(t + stride);
+        entry_next = fetch_entry(t + stride);
+        const int64_t e_word = (t * 32 + lane) * 32;
         if (e_word + 32 > n) word = (e_word < n) ? (word & ((1u << (int)(n - e_word)) - 1u)) : 0u;
+        const uint32_t seg_begin = __shfl_sync(kFullMask, entry, 0), seg_end = __shfl_sync(kFullMask, entry, 8);
+        // the step's values, from the 16-byte boundary at or below its first one
+        const uint32_t base = seg_begin & ~(uint32_t)(G - 1);
+        uint32_t nvec = (seg_end > base) ? (seg_end - base + G - 1) / G : 0u;
+        if (nvec > (uint32_t)(kSegElems / G)) nvec = kSegElems / G;   // a table that does not match the mask must not overrun the buffer
+        for (uint32_t c = lane; c < nvec; c += 32) {
+            const uint32_t e0 = base + c * G;
+            if ((int64_t)e0 + G <= k) {
+                reinterpret_cast<uint4*>(seg)[c] = ld_stream(reinterpret_cast<const uint4*>(values + e0));
+            } else {   // the last vector of `values` may be partial: element by element
+                for (int e = 0; e < G; ++e) seg[c * G + e] = ((int64_t)e0 + e < k) ? values[e0 + e] : (elem_t)0;
+            }
+        }
         const uint32_t cnt = __popc(word);
         uint32_t incl = cnt;                         // inclusive count over the lanes of this chunk (4 words)
         uint32_t up = __shfl_up_sync(kFullMask, incl, 1);
         if ((lane & 3) >= 1) incl += up;
         up = __shfl_up_sync(kFullMask, incl, 2);
         if ((lane & 3) >= 2) incl += up;
-        uint32_t pos = (w < nwords) ? __ldg(offsets + (w >> 2)) : 0u;
-        pos += incl - cnt;
+        uint32_t pos = __shfl_sync(kFullMask, entry, lane >> 2) + incl - cnt - base;   // index into the fetched piece
         const uint4 zero = make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int i = 0; i < kPitch / G; ++i) reinterpret_cast<uint4*>(img)[i * 32 + lane] = zero;
         __syncwarp();
+        // (a table that does not match the mask must not read outside the buffer)
+        if (pos + cnt > (uint32_t)kSegElems) pos = 0;
         while (word) {
             const int b = __ffs(word) - 1;
             word &= word - 1;
-            img[lane * kPitch + b] = values[pos++];
+            img[lane * kPitch + b] = seg[pos++];
         }
         __syncwarp();
         const int64_t e_tile = t * 1024;
@@ -85,11 +126,13 @@ template <typename Tr>
 static dropit_status run_decompress(const void* values, const void* meta, const uint32_t* offsets, int64_t n, int64_t k,
                                     dropit_format format, void* out, cudaStream_t stream) {
     using elem_t = typename Tr::elem_t;
+    constexpr int kDecompWarps = DecompWarps<Tr>::value;
     const int64_t cap = (int64_t)sm_count() * 16;
     if (format == DROPIT_FMT_BITMASK) {
         const int64_t ntiles = (n + 1023) / 1024;       // one warp step each
         int64_t blocks = (ntiles + kDecompWarps - 1) / kDecompWarps;
-        if (blocks > cap * 4) blocks = cap * 4;
+        const int64_t resident = (int64_t)sm_count() * kDecompCtasPerSm;   // persistent: every CTA is on an SM at once
+        if (blocks > resident) blocks = resident;
         // programmatic launch: the kernel may be brought up while the one before it drains; it waits at its top
         cudaLaunchAttribute pdl[1];
         pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -101,7 +144,7 @@ static dropit_status run_decompress(const void* values, const void* meta, const 
         cfg.attrs = pdl;
         cfg.numAttrs = 1;
         if (cudaLaunchKernelEx(&cfg, decompress_bitmask_kernel<Tr>, reinterpret_cast<const elem_t*>(values),
-                               reinterpret_cast<const uint32_t*>(meta), offsets, n, reinterpret_cast<elem_t*>(out)) !=
+                               reinterpret_cast<const uint32_t*>(meta), offsets, n, k, reinterpret_cast<elem_t*>(out)) !=
             cudaSuccess) {
             (void)cudaGetLastError();
             return DROPIT_ERR_CUDA;

@@ -78,6 +78,46 @@ def test_degenerate_tensors(cuda_device, fmt):
     _special(x, torch.float32, 0.55, fmt, cuda_device)
 
 
+# sampled (fast) path with every kind of tail: whole super-blocks, one element more, half a super-block,
+# a ragged last vector, one element short of a super-block
+TAILS = [1 << 19, (1 << 19) + 1, (1 << 19) + 512, (1 << 19) + 519, (1 << 19) + 1023, (1 << 19) + 1025,
+         148 * 32 * 1024 + 8, 148 * 32 * 2048 - 1]
+
+
+@pytest.mark.parametrize("fmt", ["bitmask", "index32"])
+@pytest.mark.parametrize("n", TAILS)
+def test_sampled_path_tails(cuda_device, n, fmt):
+    case = di.small_linear(1, n, 1, "bf16", 0.9, "gelu" if n % 2 else "normal")
+    x = di.make_x(case)
+    bits, dt, keep, k = oracle_cache(x, case.gamma)
+    cache = dropit.dropit_compress(x.to(cuda_device), case.gamma, fmt)
+    dropit.check_device_status(cuda_device)
+    assert_cache_matches_oracle(cache, bits, dt, keep, k, fmt)
+    rec = dropit.dropit_decompress(cache)
+    assert (np_bits(rec) == np.where(keep == 1, bits, 0).astype(bits.dtype)).all()
+
+
+def test_workspace_needs_no_initialisation(cuda_device):
+    """The scratch may hold anything: all ones, zeros, random bytes, or what an earlier call on another tensor left."""
+    big = di.small_linear(700, 768, 1, "bf16", 0.9)       # sampled path
+    small = di.small_linear(37, 129, 1, "bf16", 0.5)      # general path
+    xb, xs = di.make_x(big).to(cuda_device), di.make_x(small).to(cuda_device)
+    ref_b, ref_s = dropit.dropit_compress(xb, 0.9), dropit.dropit_compress(xs, 0.5)
+    nbytes = max(dropit.dropit_cache_sizes(c.n, c.gamma, dropit.BF16, dropit.FMT_BITMASK)[3] for c in (big, small))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=cuda_device)
+    g = torch.Generator(device="cpu").manual_seed(5)
+    fills = [lambda: ws.fill_(0xFF), lambda: ws.zero_(), lambda: ws.copy_(torch.randint(0, 256, (nbytes,), generator=g,
+                                                                                         dtype=torch.uint8)),
+             lambda: None, lambda: None]
+    for fill in fills:
+        fill()
+        for x, gamma, ref in ((xb, 0.9, ref_b), (xs, 0.5, ref_s), (xb, 0.9, ref_b)):
+            c = dropit.dropit_compress(x, gamma, workspace=ws)
+            assert torch.equal(c.values.view(torch.int16), ref.values.view(torch.int16))
+            assert torch.equal(c.meta, ref.meta) and torch.equal(c.offsets, ref.offsets)
+    dropit.check_device_status(cuda_device)
+
+
 def test_empty_tensor_is_a_noop(cuda_device):
     cache = dropit.dropit_compress(torch.empty(0, dtype=torch.bfloat16, device=cuda_device), 0.5)
     assert cache.k == 0 and cache.values.numel() == 0 and cache.meta.numel() == 0
