@@ -13,6 +13,10 @@
  *   - recovery R(.)        Sec. 3.2 (dropped indices filled with zero)
  *   - FC weight gradient   Eq. 6,  g = sum_{n in X_r} grad_z_j^n a_k^n ; App. A.3 G' = (A o D) x Z
  *   - conv weight gradient Eq. 4-5 (retained term), element-wise mask over the input a
+ *   - random dropping      Sec. 3.3 "Random Elements" (a gamma fraction dropped at random within the
+ *                          mini-batch): every element draws a 15-bit rank from Philox4x32-10 (Salmon,
+ *                          Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC'11) and
+ *                          the k highest ranks are retained, ties to the lower flat index
  *
  * Floating point: products and sums in double, one rounding to float at the end.
  * Elements are passed as raw bits (uint16 for bf16, uint32 for fp32); the
@@ -23,7 +27,8 @@
  * (oracle_select_rank) vs the sort (oracle_select_sort) vs numpy's stable
  * sort; closed-form keep counts; closed-form Gaussian quantiles; all-equal and
  * strictly-monotone tensors; numpy float64 matmul at gamma = 0; torch's
- * float64 conv weight gradient; 1x1 conv == FC on the transposed view.
+ * float64 conv weight gradient; 1x1 conv == FC on the transposed view; the
+ * Philox test vectors printed with the generator's reference distribution.
  */
 #include <math.h>
 #include <stdint.h>
@@ -32,6 +37,42 @@
 
 #define DT_BF16 0
 #define DT_F32 1
+
+/* ---- random ranks (Sec. 3.3 "Random Elements") -------------------------- */
+
+/* Philox4x32-10 as published (SC'11, Sec. 3.3 / Table 2 of that paper): ten rounds of
+ *   (c0, c1, c2, c3) <- (hi(M1*c2) ^ c1 ^ k0,  lo(M1*c2),  hi(M0*c0) ^ c3 ^ k1,  lo(M0*c0)),
+ * the key (k0, k1) raised by the Weyl constants (W0, W1) between rounds. */
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        const uint64_t p0 = (uint64_t)M0 * c0, p1 = (uint64_t)M1 * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += W0;
+        k1 += W1;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* Rank of element i under seed s: block b = i div 8 is the counter (b_lo, b_hi, 0, 0), the seed is the
+ * key (s_lo, s_hi); the four output words hold eight 16-bit halves, low half first, and element i takes
+ * half (i mod 8) without its top bit (15 bits). */
+void oracle_random_ranks(int64_t n, uint64_t seed, uint32_t* ranks) {
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    for (int64_t i = 0; i < n; ++i) {
+        const uint64_t b = (uint64_t)i / 8;
+        const uint32_t ctr[4] = {(uint32_t)b, (uint32_t)(b >> 32), 0u, 0u};
+        uint32_t out[4];
+        oracle_philox4x32_10(ctr, key, out);
+        const int e = (int)(i % 8);
+        ranks[i] = (out[e / 2] >> (16 * (e % 2))) & 0x7FFFu;
+    }
+}
 
 /* ---- element decoding ------------------------------------------------- */
 
@@ -138,6 +179,20 @@ int oracle_min_k(const void* x, int64_t n, double gamma, int dtype, uint8_t* kee
 
 /* Occupancy bitmask: element i <-> bit (i mod 32) of 32-bit word (i div 32);
  * the unused high bits of the last word are 0.  words has ceil(n/32) entries. */
+/* D(.) with the random strategy (Sec. 3.3 "Random Elements"): the same number of elements is retained as
+ * under min-k, chosen by rank instead of magnitude. */
+int oracle_random_k(int64_t n, double gamma, uint64_t seed, uint8_t* keep, int64_t* k_out) {
+    const int64_t k = oracle_keep_count(n, gamma);
+    if (k_out) *k_out = k;
+    if (n <= 0) return 0;
+    uint32_t* ranks = (uint32_t*)malloc((size_t)n * sizeof(uint32_t));
+    if (!ranks) return -1;
+    oracle_random_ranks(n, seed, ranks);
+    const int rc = oracle_select_sort(ranks, n, k, keep);
+    free(ranks);
+    return rc;
+}
+
 void oracle_encode_bitmask(const uint8_t* keep, int64_t n, uint32_t* words) {
     int64_t nw = (n + 31) / 32;
     for (int64_t w = 0; w < nw; ++w) words[w] = 0;

@@ -17,7 +17,7 @@ __all__ = [
     "BF16", "F32", "build", "to_bits", "keep_count", "keys", "select_rank", "select_sort", "min_k",
     "encode_bitmask", "encode_index32", "pack_values", "chunk_offsets", "recover_from_bitmask",
     "recover_from_index32", "fc_weight_grad", "fc_weight_grad_entries", "conv_weight_grad",
-    "conv_weight_grad_entries", "num_threads", "bits_to_float64",
+    "conv_weight_grad_entries", "num_threads", "bits_to_float64", "philox4x32_10", "random_ranks", "random_k",
 ]
 
 BF16 = 0
@@ -51,6 +51,7 @@ def _load():
             lib.oracle_pack_values.restype = ctypes.c_int64
             lib.oracle_select_sort.restype = ctypes.c_int
             lib.oracle_min_k.restype = ctypes.c_int
+            lib.oracle_random_k.restype = ctypes.c_int
             lib.oracle_num_threads.restype = ctypes.c_int
             _lib = lib
     return _lib
@@ -138,6 +139,34 @@ def min_k(x_bits: np.ndarray, gamma: float, dtype: int):
                               ctypes.byref(k))
     if rc != 0:
         raise MemoryError("oracle_min_k")
+    return keep, int(k.value)
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """One block of Philox4x32-10 (Salmon et al., SC'11): 4 counter words, 2 key words -> 4 output words."""
+    c = np.ascontiguousarray(ctr, np.uint32)
+    k = np.ascontiguousarray(key, np.uint32)
+    assert c.size == 4 and k.size == 2
+    out = np.empty(4, np.uint32)
+    _load().oracle_philox4x32_10(_p(c), _p(k), _p(out))
+    return out
+
+
+def random_ranks(n: int, seed: int) -> np.ndarray:
+    """15-bit rank of every element under `seed` (Sec. 3.3 "Random Elements")."""
+    out = np.empty(int(n), np.uint32)
+    _load().oracle_random_ranks(_i64(n), ctypes.c_uint64(int(seed) & (2 ** 64 - 1)), _p(out))
+    return out
+
+
+def random_k(n: int, gamma: float, seed: int):
+    """D(.) with the random strategy (Sec. 3.3): the k highest ranks stay -> (keep uint8[n], k)."""
+    keep = np.empty(int(n), np.uint8)
+    k = ctypes.c_int64(0)
+    rc = _load().oracle_random_k(_i64(n), ctypes.c_double(gamma), ctypes.c_uint64(int(seed) & (2 ** 64 - 1)), _p(keep),
+                                 ctypes.byref(k))
+    if rc != 0:
+        raise MemoryError("oracle_random_k")
     return keep, int(k.value)
 
 
