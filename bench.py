@@ -117,6 +117,20 @@ def dense_flops(case) -> float:
     return 2.0 * case.M * case.Ca * case.Cz
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """A multi-rank time is the slowest rank's device time."""
+    if world > 1:
+        t = torch.tensor([ms], device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def whole_job_value(world: int, steps: int, ms: float) -> float:
+    """Samples per second of all ranks together (every rank runs the same step on its own batch: weak scaling)."""
+    return world * BATCH_IMAGES * steps / (ms / 1e3)
+
+
 def run_ours(args, rank, world, device):
     import paper_2202_13808_b200 as dropit
 
@@ -172,11 +186,7 @@ def run_ours(args, rank, world, device):
     launches = dropit.dropit_launch_count() - launches0
     clocks = sampler.stop(t0, t1) if rank == 0 else None
     dropit.check_device_status(device)
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=device)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), world, device)
 
     comp_ms = [statistics.mean(evs[i][li][0].elapsed_time(evs[i][li][1]) for i in range(args.steps)) for li in range(2)]
     dw_ms = [statistics.mean(evs[i][li][1].elapsed_time(evs[i][li][2]) for i in range(args.steps)) for li in range(2)]
@@ -206,17 +216,13 @@ def run_ours(args, rank, world, device):
         e2e_step()
     f1.record(stream)
     barrier()
-    e2e_ms = f0.elapsed_time(f1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=device)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(f0.elapsed_time(f1), world, device)
 
     if rank != 0:
         return None
     peaks = measured_peaks()
     ms_per_step = ms / args.steps
-    value = world * BATCH_IMAGES * args.steps / (ms / 1e3)
+    value = whole_job_value(world, args.steps, ms)
     # dominant kernel: the fc weight-gradient GEMM (both layers have the same flop count)
     F = dense_flops(LAYERS[0])
     dw_avg_ms = statistics.mean(dw_ms)
@@ -246,7 +252,7 @@ def run_ours(args, rank, world, device):
                                               "frac": comp_gbs[0] / peaks["hbm_gbs"], "avg_ms": comp_ms[0]}},
         "per_call_ms": {"compress_fc1": comp_ms[0], "compress_fc2": comp_ms[1], "dw_fc1": dw_ms[0], "dw_fc2": dw_ms[1]},
         "dw_tflops": {"fc1": F / (dw_ms[0] * 1e-3) / 1e12, "fc2": F / (dw_ms[1] * 1e-3) / 1e12},
-        "e2e": {"value": world * BATCH_IMAGES * e2e_steps / (e2e_ms / 1e3), "unit": "samples/s",
+        "e2e": {"value": whole_job_value(world, e2e_steps, e2e_ms), "unit": "samples/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches),
         "clocks": clocks,
