@@ -111,6 +111,28 @@ dropit_status dropit_compress(const void* x, int64_t n, double gamma, dropit_dty
                               void* values, void* meta, uint32_t* offsets, void* workspace, size_t workspace_bytes,
                               int32_t* dev_status, void* cuda_stream);
 
+/*
+ * D(a) with the RANDOM strategy (Sec. 3.3 "Random Elements": a gamma fraction of
+ * the elements is dropped at random within the mini-batch; the baseline of
+ * Table 2).  The paper does not say how the random set is drawn; here exactly
+ * k = dropit_keep_count(n, gamma) elements are retained, as under min-k, so the
+ * cache has the same size: element i draws a 15-bit rank from Philox4x32-10
+ * (Salmon et al., SC'11; the 64-bit block index i div 8 fills the first two
+ * counter words, the other two are 0, key = seed; the four output words are
+ * eight 16-bit halves, low half first, and element i takes half i mod 8
+ * without its top bit), and the k highest ranks stay, ties to the lower flat
+ * index.  With 15-bit ranks the elements that share the threshold rank (about
+ * n / 32768 of them) are the only ones whose fate depends on their position.
+ * The retained set depends on (n, gamma, seed) only, never on the data.
+ * Same cache layout and arguments as dropit_compress; workspace of at least
+ * dropit_compress_random_workspace bytes (it holds the ranks: about 2 bytes per
+ * element), contents destroyed, need not be initialised.
+ */
+dropit_status dropit_compress_random_workspace(int64_t n, double gamma, size_t* workspace_bytes);
+dropit_status dropit_compress_random(const void* x, int64_t n, double gamma, uint64_t seed, dropit_dtype dtype,
+                                     dropit_format format, void* values, void* meta, uint32_t* offsets,
+                                     void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
 /* Largest tensor (elements) that dropit_compress_static accepts. */
 #define DROPIT_STATIC_MAX_ELEMS (1 << 28)
 

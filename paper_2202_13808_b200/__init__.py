@@ -7,7 +7,7 @@ There is no CPU or eager fallback.
 """
 from .api import (  # noqa: F401
     BF16, F32, FMT_BITMASK, FMT_INDEX32, CHUNK, DropITCache, DropITError,
-    dropit_cache_sizes, dropit_compress, dropit_conv_weight_grad, dropit_conv_weight_grad_workspace,
+    dropit_cache_sizes, dropit_compress, dropit_compress_random, dropit_compress_random_workspace, dropit_conv_weight_grad, dropit_conv_weight_grad_workspace,
     dropit_decompress, dropit_keep_count, dropit_launch_count, dropit_status_string, dropit_version, dropit_weight_grad,
     dropit_weight_grad_workspace, check_device_status, library_path,
 )

@@ -150,6 +150,39 @@ def dropit_compress(x: torch.Tensor, gamma: float, fmt="bitmask", workspace: Opt
     return DropITCache(values, meta, offsets, n, k, tuple(x.shape), x.dtype, fmt, float(gamma))
 
 
+@functools.lru_cache(maxsize=4096)
+def dropit_compress_random_workspace(n: int, gamma: float) -> int:
+    out = ctypes.c_size_t(0)
+    _check(_lib.load().dropit_compress_random_workspace(int(n), float(gamma), ctypes.byref(out)),
+           "dropit_compress_random_workspace")
+    return int(out.value)
+
+
+def dropit_compress_random(x: torch.Tensor, gamma: float, seed: int, fmt="bitmask",
+                           workspace: Optional[torch.Tensor] = None) -> DropITCache:
+    """D(a), random strategy (Sec. 3.3 "Random Elements"): k elements chosen by Philox rank under `seed`."""
+    _require_cuda(x, "x")
+    lib = _lib.load()
+    fmt = _FMT_CODE[fmt]
+    dt = _DTYPE_CODE[x.dtype]
+    n = x.numel()
+    vb, mb, ob, _ = dropit_cache_sizes(n, gamma, dt, fmt)
+    wb = dropit_compress_random_workspace(n, gamma)
+    k = dropit_keep_count(n, gamma)
+    dev = x.device
+    values = torch.empty(vb // x.element_size(), dtype=x.dtype, device=dev)
+    meta = torch.empty(mb // 4, dtype=torch.int32, device=dev)
+    offsets = torch.empty(ob // 4, dtype=torch.int32, device=dev)
+    if workspace is None or workspace.numel() < wb:
+        workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
+    with _on_device(dev):
+        code = lib.dropit_compress_random(_ptr(x), n, float(gamma), int(seed) & (2 ** 64 - 1), dt, fmt, _ptr(values),
+                                          _ptr(meta), _ptr(offsets), _ptr(workspace), workspace.numel(),
+                                          _ptr(_status_word(dev)), _stream_ptr(dev))
+    _check(code, "dropit_compress_random")
+    return DropITCache(values, meta, offsets, n, k, tuple(x.shape), x.dtype, fmt, float(gamma))
+
+
 def dropit_decompress(cache: DropITCache) -> torch.Tensor:
     """R(a-hat) (Sec. 3.2): dense tensor, dropped positions +0."""
     lib = _lib.load()

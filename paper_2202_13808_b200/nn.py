@@ -21,6 +21,13 @@ import torch.nn.functional as F
 from . import api
 
 
+def _compress(x: torch.Tensor, gamma: float, fmt: str, seed):
+    """Min-k (seed None) or random (an integer seed) compression of a layer input: the two strategies of Sec. 3.3."""
+    if seed is None:
+        return api.dropit_compress(x, gamma, fmt)
+    return api.dropit_compress_random(x, gamma, int(seed), fmt)
+
+
 def _check_input(x: torch.Tensor):
     if not x.is_cuda:
         raise ValueError("DropIT layers need CUDA tensors (there is no CPU path)")
@@ -32,7 +39,7 @@ class DropITLinearFn(torch.autograd.Function):
     """y = x W^T + b with the cached x replaced by its min-k compression."""
 
     @staticmethod
-    def forward(ctx, x, weight, bias, gamma: float, fmt: str):
+    def forward(ctx, x, weight, bias, gamma: float, fmt: str, seed=None):
         _check_input(x)
         z = F.linear(x, weight, bias)
         ctx.has_bias = bias is not None
@@ -42,7 +49,7 @@ class DropITLinearFn(torch.autograd.Function):
             x2 = x.reshape(-1, x.shape[-1])
             if not x2.is_contiguous():
                 x2 = x2.contiguous()
-            cache = api.dropit_compress(x2, gamma, fmt)
+            cache = _compress(x2, gamma, fmt, seed)
             ctx.cache_meta = (cache.n, cache.k, cache.shape, cache.dtype, cache.fmt, cache.gamma)
             ctx.save_for_backward(weight, cache.values, cache.meta, cache.offsets)
         else:
@@ -66,14 +73,14 @@ class DropITLinearFn(torch.autograd.Function):
             dw = api.dropit_weight_grad(dzc, cache).to(weight.dtype)   # Eq. 6
         if ctx.has_bias and ctx.needs_input_grad[2]:
             db = dz2.sum(0)
-        return dx, dw, db, None, None
+        return dx, dw, db, None, None, None
 
 
 class DropITConv2dFn(torch.autograd.Function):
     """Conv2d (groups 1, dilation 1) with the cached input replaced by its min-k compression."""
 
     @staticmethod
-    def forward(ctx, x, weight, bias, stride: int, padding: int, gamma: float, fmt: str):
+    def forward(ctx, x, weight, bias, stride: int, padding: int, gamma: float, fmt: str, seed=None):
         _check_input(x)
         z = F.conv2d(x, weight, bias, stride=stride, padding=padding)
         ctx.has_bias = bias is not None
@@ -82,7 +89,7 @@ class DropITConv2dFn(torch.autograd.Function):
         ctx.cache_meta = None
         if weight.requires_grad:
             xc = x if x.is_contiguous() else x.contiguous()
-            cache = api.dropit_compress(xc, gamma, fmt)
+            cache = _compress(xc, gamma, fmt, seed)
             ctx.cache_meta = (cache.n, cache.k, cache.shape, cache.dtype, cache.fmt, cache.gamma)
             ctx.save_for_backward(weight, cache.values, cache.meta, cache.offsets)
         else:
@@ -106,27 +113,45 @@ class DropITConv2dFn(torch.autograd.Function):
                                              ctx.padding).to(weight.dtype)   # Eq. 4-5
         if ctx.has_bias and ctx.needs_input_grad[2]:
             db = dz.sum((0, 2, 3))
-        return dx, dw, db, None, None, None, None
+        return dx, dw, db, None, None, None, None, None
 
 
-class DropITLinear(nn.Linear):
-    """nn.Linear whose backward uses a min-k compressed input cache. `gamma` is the dropped fraction."""
+class _Strategy:
+    """Dropping strategy of a layer (Sec. 3.3): "min_k", or "random" with a seed that advances by one per call."""
 
-    def __init__(self, in_features, out_features, bias=True, gamma: float = 0.9, fmt: str = "bitmask", **kw):
+    def _init_strategy(self, strategy: str, seed: int):
+        if strategy not in ("min_k", "random"):
+            raise ValueError("strategy must be 'min_k' or 'random'")
+        self.strategy, self.seed, self._calls = strategy, int(seed), 0
+
+    def _next_seed(self):
+        if self.strategy == "min_k":
+            return None
+        self._calls += 1
+        return self.seed + self._calls - 1
+
+
+class DropITLinear(nn.Linear, _Strategy):
+    """nn.Linear whose backward uses a compressed input cache. `gamma` is the dropped fraction."""
+
+    def __init__(self, in_features, out_features, bias=True, gamma: float = 0.9, fmt: str = "bitmask",
+                 strategy: str = "min_k", seed: int = 0, **kw):
         super().__init__(in_features, out_features, bias=bias, **kw)
         self.gamma, self.fmt = float(gamma), fmt
+        self._init_strategy(strategy, seed)
 
     def forward(self, x):
         if not (self.training and torch.is_grad_enabled()):
             return F.linear(x, self.weight, self.bias)     # inference is unchanged (Sec. 3.5)
-        return DropITLinearFn.apply(x, self.weight, self.bias, self.gamma, self.fmt)
+        return DropITLinearFn.apply(x, self.weight, self.bias, self.gamma, self.fmt, self._next_seed())
 
 
-class DropITConv2d(nn.Conv2d):
-    """nn.Conv2d (groups 1, dilation 1, square stride/padding) with a min-k compressed input cache."""
+class DropITConv2d(nn.Conv2d, _Strategy):
+    """nn.Conv2d (groups 1, dilation 1, square stride/padding) with a compressed input cache."""
 
-    def __init__(self, *args, gamma: float = 0.8, fmt: str = "bitmask", **kw):
+    def __init__(self, *args, gamma: float = 0.8, fmt: str = "bitmask", strategy: str = "min_k", seed: int = 0, **kw):
         super().__init__(*args, **kw)
+        self._init_strategy(strategy, seed)
         if self.groups != 1 or self.dilation != (1, 1) or self.stride[0] != self.stride[1] or \
                 self.padding[0] != self.padding[1] or self.padding_mode != "zeros":
             raise ValueError("DropITConv2d supports groups=1, dilation=1, square stride and zero padding")
@@ -135,7 +160,8 @@ class DropITConv2d(nn.Conv2d):
     def forward(self, x):
         if not (self.training and torch.is_grad_enabled()):
             return F.conv2d(x, self.weight, self.bias, self.stride, self.padding)
-        return DropITConv2dFn.apply(x, self.weight, self.bias, self.stride[0], self.padding[0], self.gamma, self.fmt)
+        return DropITConv2dFn.apply(x, self.weight, self.bias, self.stride[0], self.padding[0], self.gamma, self.fmt,
+                                    self._next_seed())
 
 
 def convert_linear_layers(module: nn.Module, gamma: float, fmt: str = "bitmask",

@@ -31,6 +31,8 @@ def _algorithmic(case, op):
     n = case.n
     es = 2 if case.dtype == "bf16" else 4
     k = dropit.dropit_keep_count(n, case.gamma)
+    if op == "compress_random":   # ranks written once and read twice (2 bytes each), retained x gathered, outputs
+        return 3 * n * 2 + n / 8 + 2 * k * es + 4 * ((n + 127) // 128), 0.0
     if op == "compress":
         passes = 2 if es == 2 else 3
         return passes * n * es + n / 8 + k * es + 4 * ((n + 127) // 128), 0.0
@@ -43,7 +45,7 @@ def _algorithmic(case, op):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["compress", "decompress", "weight_grad", "conv_weight_grad"])
+    ap.add_argument("op", choices=["compress", "compress_random", "decompress", "weight_grad", "conv_weight_grad"])
     ap.add_argument("case", choices=sorted(CASES))
     ap.add_argument("--gamma", type=float, default=None)
     ap.add_argument("--format", default="bitmask", choices=["bitmask", "index32"])
@@ -67,6 +69,8 @@ def main():
         b = i % nsets
         if args.op == "compress":
             caches[b] = dropit.dropit_compress(xs[b], gamma, args.format)
+        elif args.op == "compress_random":
+            caches[b] = dropit.dropit_compress_random(xs[b], gamma, i, args.format)
         elif args.op == "decompress":
             dropit.dropit_decompress(caches[b])
         elif args.op == "weight_grad":
