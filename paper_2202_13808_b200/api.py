@@ -183,11 +183,14 @@ def dropit_compress_random(x: torch.Tensor, gamma: float, seed: int, fmt="bitmas
     return DropITCache(values, meta, offsets, n, k, tuple(x.shape), x.dtype, fmt, float(gamma))
 
 
-def dropit_decompress(cache: DropITCache) -> torch.Tensor:
-    """R(a-hat) (Sec. 3.2): dense tensor, dropped positions +0."""
+def dropit_decompress(cache: DropITCache, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """R(a-hat) (Sec. 3.2): dense tensor, dropped positions +0; written into `out` when given."""
     lib = _lib.load()
     dev = cache.offsets.device if cache.offsets.numel() else cache.values.device
-    out = torch.empty(cache.shape, dtype=cache.dtype, device=dev)
+    if out is None:
+        out = torch.empty(cache.shape, dtype=cache.dtype, device=dev)
+    elif out.numel() != cache.n or out.dtype != cache.dtype or not out.is_contiguous() or out.device != dev:
+        raise ValueError("out must be a contiguous %s tensor of %d elements on %s" % (cache.dtype, cache.n, dev))
     with _on_device(dev):
         code = lib.dropit_decompress(_ptr(cache.values), _ptr(cache.meta), _ptr(cache.offsets), cache.n, cache.k,
                                      _DTYPE_CODE[cache.dtype], cache.fmt, _ptr(out), _stream_ptr(dev))
