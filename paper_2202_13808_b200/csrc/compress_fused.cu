@@ -190,6 +190,7 @@ __device__ __forceinline__ void phase_stamp(FusedState*, int) {}
 template <typename AfterLoads>
 __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t n, unsigned long long k, uint32_t* bins,
                                             uint32_t* s_warp, uint32_t* band, FusedState* st, AfterLoads after_loads) {
+    // after_loads: called once by every thread, after the sample has been counted (or at once when there is no sample)
     const int64_t nvec = n / 8;
     const bool sampled = n >= kSampleMinElems;
     uint4 sv[kSampleVecs / kFusedThreads];
@@ -202,7 +203,7 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
             sv[r] = ld_stream(x + (int64_t)s * stride + (int64_t)(h % (uint32_t)stride));
         }
     }
-    after_loads();   // whatever the caller wants in flight behind the sample loads
+    if (!sampled) after_loads();
     if (threadIdx.x == 0) {
         band[0] = 0;
         band[1] = kKeySpace - 1;
@@ -222,6 +223,7 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
         }
         __syncthreads();
         phase_stamp(st, 9);
+        after_loads();   // what the caller wants in flight while the thresholds are worked out (issued earlier, it delays the sample)
         // ranks (counted from the largest key) that bracket the threshold with a 6-sigma margin
         const float S = (float)(kSampleVecs * 8);
         const float p = (float)((double)k / (double)n);
@@ -478,7 +480,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         st->n_hi[1] = 0;
     }
     barrier_open(&st->barrier, epoch);
-    // the first blocks of the run are requested right behind the sample loads, whose processing hides their latency
+    // the first super-block of the run is requested while the sample is evaluated, which hides its latency
     bool prefetched = true;
     sample_band(x, n, k, sample_bins, sh.warp, sh.band, st, [&] { issue_sb(sb0, 0); });
     uint32_t lo = sh.band[0], hi = sh.band[1];
