@@ -223,13 +223,15 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
         }
         __syncthreads();
         phase_stamp(st, 9);
-        after_loads();   // what the caller wants in flight while the thresholds are worked out (issued earlier, it delays the sample)
         // ranks (counted from the largest key) that bracket the threshold with a 6-sigma margin
         const float S = (float)(kSampleVecs * 8);
         const float p = (float)((double)k / (double)n);
         const float ks = p * S;
         const float margin = 6.0f * sqrtf(S * p * (1.0f - p)) + 16.0f;
         const float r_hi = ks - margin, r_lo = ks + margin;
+        // as integers: for an integer count c, c < r <=> c < ceil(r) and r <= c <=> ceil(r) <= c.  0 = no such rank.
+        const uint32_t R_hi = (r_hi >= 1.0f) ? (uint32_t)ceilf(r_hi) : 0u;
+        const uint32_t R_lo = (r_lo <= S) ? (uint32_t)ceilf(r_lo) : 0u;
         constexpr int PER = kKeySpace / kFusedThreads;   // keys per thread, descending: kKeySpace-1 - (t*PER + r)
         const int t = threadIdx.x;
         static_assert(PER == 32, "the walk below assumes 16 words per thread");
@@ -243,6 +245,7 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
                 cw[4 * j] = v.x; cw[4 * j + 1] = v.y; cw[4 * j + 2] = v.z; cw[4 * j + 3] = v.w;
             }
         }
+        after_loads();   // what the caller wants in flight while the thresholds are worked out (issued earlier, it delays the sample)
         uint32_t sum = 0;
 #pragma unroll
         for (int r = 0; r < PER / 2; ++r) sum += (cw[r] & 0xFFFFu) + (cw[r] >> 16);
@@ -250,8 +253,7 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
         const uint32_t excl = block_exclusive_scan(sum, s_warp, &total);
         phase_stamp(st, 10);
         // key at descending rank r: cum_before < r <= cum_before + h
-        if ((r_hi >= 1.0f && (float)excl < r_hi && r_hi <= (float)(excl + sum)) ||
-            (r_lo <= S && (float)excl < r_lo && r_lo <= (float)(excl + sum))) {
+        if ((excl < R_hi && R_hi <= excl + sum) || (excl < R_lo && R_lo <= excl + sum)) {
             uint32_t cum = excl;
 #pragma unroll
             for (int r = 0; r < PER; ++r) {
@@ -259,10 +261,8 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
                 const uint32_t key = kKeySpace - 1 - (t * PER + r);
                 const uint32_t cwr = cw[PER / 2 - 1 - r / 2];
                 const uint32_t hh = (r & 1) ? (cwr & 0xFFFFu) : (cwr >> 16);
-                if (hh) {
-                    if (r_hi >= 1.0f && (float)cum < r_hi && r_hi <= (float)(cum + hh)) band[1] = key;
-                    if (r_lo <= S && (float)cum < r_lo && r_lo <= (float)(cum + hh)) band[0] = key;
-                }
+                if (cum < R_hi && R_hi <= cum + hh) band[1] = key;
+                if (cum < R_lo && R_lo <= cum + hh) band[0] = key;
                 cum += hh;
             }
         }
