@@ -404,13 +404,16 @@ __device__ __forceinline__ void sb_issue_full(uint32_t lane_slot, const uint4* s
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(lane_slot + j * 512), "l"(src + j * 32) : "memory");
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
-// The lane's 32 elements (16 words) of a slot; `own` = shared address of the slot + 64 * lane.
-__device__ __forceinline__ void sb_read(uint32_t own, uint32_t (&w)[16]) {
+// The lane's 32 elements (16 words) of a slot; `own` = shared address of the slot + 64 * lane.  The lanes of a
+// warp read 64-byte pieces 64 bytes apart, which would put every other lane of a quarter-warp on the same banks;
+// so the lane's j-th load takes its vector j ^ rot (rot = (lane / 2) % 4) and the eight lanes of a quarter-warp
+// touch eight different 16-byte columns.  w[4 * j ..] then holds the lane's elements 8 * (j ^ rot) ..
+__device__ __forceinline__ void sb_read(uint32_t own, uint32_t rot, uint32_t (&w)[16]) {
 #pragma unroll
     for (int j = 0; j < 4; ++j)
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
                      : "=r"(w[4 * j]), "=r"(w[4 * j + 1]), "=r"(w[4 * j + 2]), "=r"(w[4 * j + 3])
-                     : "r"(own + j * 16)
+                     : "r"(own + ((j ^ rot) << 4))
                      : "memory");
 }
 // All but the most recently committed super-block have landed.
@@ -456,6 +459,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     const uint32_t ring_warp = ptx_smem(fsm) + warp * (kRingSlots * kSbBytes);
     const uint32_t ring_copy = ring_warp + lane * 16;   // where the lane's copies of a slot start
     const uint32_t ring_own = ring_warp + lane * 64;    // the lane's 32 elements of a slot
+    const uint32_t rot = (uint32_t)(lane >> 1) & 3u;     // see sb_read
     const int64_t nvec_full = n / 8;
     const int64_t blocks_total = (n + kBlkElems - 1) / kBlkElems;
     const int64_t blk0 = ((int64_t)blockIdx.x * kFusedWarps + warp) * blocks_per_warp;   // even
@@ -549,7 +553,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                 __syncwarp();   // the lane reads vectors that other lanes copied
                 const uint32_t own = ring_own + slot * kSbBytes;
                 uint32_t w[16];
-                sb_read(own, w);
+                sb_read(own, rot, w);
                 uint32_t hi_flags = 0, pending = 0;
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {   // four words = eight elements at a time
@@ -563,7 +567,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                     // above the band only the count matters: the flag bytes of all 16 words share one word
                     hi_flags |= ((__byte_perm(a[0], a[1], 0x7531) & 0x80808080u) >> (2 * g)) |
                                 ((__byte_perm(a[2], a[3], 0x7531) & 0x80808080u) >> (2 * g + 1));
-                    pending |= flags8(b[0], b[1], b[2], b[3]) << (8 * g);
+                    pending |= flags8(b[0], b[1], b[2], b[3]) << ((g ^ rot) << 3);
                 }
                 cnt_hi += __popc(hi_flags);
                 if constexpr (!FULL) pending &= valid_mask32(sb * kSbElems + lane * 32, n);   // zero padding is no data
@@ -860,7 +864,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         uint32_t g32 = 0, ge32 = 0;
         {
             uint32_t w[16];
-            sb_read(own, w);
+            sb_read(own, rot, w);
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 uint32_t a[4], b[4];
@@ -870,8 +874,8 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                     a[i] = m + c_gt;                       // bit 15 of a half: key > T
                     b[i] = m + c_ge;                       // bit 15 of a half: key >= T
                 }
-                g32 |= flags8(a[0], a[1], a[2], a[3]) << (8 * g);
-                ge32 |= flags8(b[0], b[1], b[2], b[3]) << (8 * g);
+                g32 |= flags8(a[0], a[1], a[2], a[3]) << ((g ^ rot) << 3);
+                ge32 |= flags8(b[0], b[1], b[2], b[3]) << ((g ^ rot) << 3);
             }
         }
         uint32_t e32 = ge32 & ~g32;   // key == T
