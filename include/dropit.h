@@ -156,7 +156,8 @@ dropit_status dropit_compress_random(const void* x, int64_t n, double gamma, uin
  *    up the array's device address (with that device current); make that first
  *    call outside any stream capture.
  *  - All calls on a device share the one array, and it keeps whatever the last
- *    call left there; each call clears the part that must start at zero itself.
+ *    call left there; each call resets, when its kernel starts, the few words
+ *    that must start fresh (its counters and its barrier word).
  *    Two calls that overlap on the GPU (different streams, no ordering between
  *    them) would trample each other's scratch: order them.
  */

@@ -118,6 +118,20 @@ def test_workspace_needs_no_initialisation(cuda_device):
     dropit.check_device_status(cuda_device)
 
 
+def test_decompress_into_a_given_buffer(cuda_device):
+    case = di.small_linear(300, 3072, 1, "bf16", 0.9, "gelu")
+    x = di.make_x(case).to(cuda_device)
+    cache = dropit.dropit_compress(x, case.gamma)
+    out = torch.full((case.n,), float("nan"), dtype=torch.bfloat16, device=cuda_device)
+    got = dropit.dropit_decompress(cache, out=out)
+    assert got.data_ptr() == out.data_ptr()
+    assert torch.equal(out.view(torch.int16), dropit.dropit_decompress(cache).reshape(-1).view(torch.int16))
+    with pytest.raises(ValueError):
+        dropit.dropit_decompress(cache, out=torch.empty(case.n - 1, dtype=torch.bfloat16, device=cuda_device))
+    with pytest.raises(ValueError):
+        dropit.dropit_decompress(cache, out=torch.empty(case.n, dtype=torch.float32, device=cuda_device))
+
+
 def test_empty_tensor_is_a_noop(cuda_device):
     cache = dropit.dropit_compress(torch.empty(0, dtype=torch.bfloat16, device=cuda_device), 0.5)
     assert cache.k == 0 and cache.values.numel() == 0 and cache.meta.numel() == 0
