@@ -97,6 +97,32 @@ def test_sampled_path_tails(cuda_device, n, fmt):
     assert (np_bits(rec) == np.where(keep == 1, bits, 0).astype(bits.dtype)).all()
 
 
+@pytest.mark.parametrize("fmt", ["bitmask", "index32"])
+def test_degenerate_tensors_on_the_sampled_path(cuda_device, fmt):
+    """Large tensors (sampled band, per-warp histograms) whose threshold sits in a huge tie."""
+    n = (1 << 20) + 777
+    rng = np.random.default_rng(11)
+    # ReLU-like: half exact zeros, and more elements to retain than there are non-zeros: T = 0, the quota ends among the zeros
+    x = np.abs(rng.standard_normal(n)).astype(np.float32)
+    x[rng.random(n) < 0.5] = 0.0
+    bits = (x.view(np.uint32) >> 16).astype(np.uint16)
+    bits[::7] |= 0x8000                                   # some -0 and negative values
+    _special(bits, torch.bfloat16, 0.3, fmt, cuda_device)
+    # all equal magnitude: the lowest indices win
+    x = np.full(n, 0x3F80, np.uint16); x[::2] |= 0x8000
+    keep = _special(x, torch.bfloat16, 0.7, fmt, cuda_device)
+    k = int(keep.sum()); assert keep[:k].all() and not keep[k:].any()
+    # three distinct magnitudes
+    x = rng.integers(0, 3, n).astype(np.uint16) * 0x0100 + 0x3F00
+    _special(x, torch.bfloat16, 0.55, fmt, cuda_device)
+    # a few huge outliers (Inf, NaN patterns) in Gaussian data
+    x = (rng.standard_normal(n).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    x[rng.integers(0, n, 50)] = 0x7F80
+    x[rng.integers(0, n, 50)] = 0x7FC1
+    _special(x, torch.bfloat16, 0.9, fmt, cuda_device)
+    _special(x, torch.bfloat16, 0.999, fmt, cuda_device)
+
+
 def test_workspace_needs_no_initialisation(cuda_device):
     """The scratch may hold anything: all ones, zeros, random bytes, or what an earlier call on another tensor left."""
     big = di.small_linear(700, 768, 1, "bf16", 0.9)       # sampled path
