@@ -235,25 +235,29 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
         constexpr int PER = kKeySpace / kFusedThreads;   // keys per thread, descending: kKeySpace-1 - (t*PER + r)
         const int t = threadIdx.x;
         static_assert(PER == 32, "the walk below assumes 16 words per thread");
-        // the thread's 16 words, kept in registers for the walk below
-        uint32_t cw[PER / 2];
-        {
-            const uint4* mine = reinterpret_cast<const uint4*>(bins + (kKeySpace / 2 - (t + 1) * (PER / 2)));
-#pragma unroll
-            for (int j = 0; j < PER / 8; ++j) {
-                const uint4 v = mine[j];
-                cw[4 * j] = v.x; cw[4 * j + 1] = v.y; cw[4 * j + 2] = v.z; cw[4 * j + 3] = v.w;
-            }
-        }
-        after_loads();   // what the caller wants in flight while the thresholds are worked out (issued earlier, it delays the sample)
+        // the thread's 16 words hold its 32 counters; the four 16-byte reads go in an order rotated by (t/2) mod 4,
+        // so that the threads of a quarter-warp (64 bytes apart) touch different banks
+        const uint4* mine = reinterpret_cast<const uint4*>(bins + (kKeySpace / 2 - (t + 1) * (PER / 2)));
         uint32_t sum = 0;
 #pragma unroll
-        for (int r = 0; r < PER / 2; ++r) sum += (cw[r] & 0xFFFFu) + (cw[r] >> 16);
+        for (int j = 0; j < PER / 8; ++j) {
+            const uint4 v = mine[j ^ ((t >> 1) & 3)];
+            sum += (v.x & 0xFFFFu) + (v.x >> 16) + (v.y & 0xFFFFu) + (v.y >> 16) + (v.z & 0xFFFFu) + (v.z >> 16) +
+                   (v.w & 0xFFFFu) + (v.w >> 16);
+        }
+        after_loads();   // what the caller wants in flight while the thresholds are worked out (issued earlier, it delays the sample)
         uint32_t total;
         const uint32_t excl = block_exclusive_scan(sum, s_warp, &total);
         phase_stamp(st, 10);
         // key at descending rank r: cum_before < r <= cum_before + h
         if ((excl < R_hi && R_hi <= excl + sum) || (excl < R_lo && R_lo <= excl + sum)) {
+            // one or two threads of the CTA get here: they read their counters again, in key order
+            uint32_t cw[PER / 2];
+#pragma unroll
+            for (int j = 0; j < PER / 8; ++j) {
+                const uint4 v = mine[j];
+                cw[4 * j] = v.x; cw[4 * j + 1] = v.y; cw[4 * j + 2] = v.z; cw[4 * j + 3] = v.w;
+            }
             uint32_t cum = excl;
 #pragma unroll
             for (int r = 0; r < PER; ++r) {
