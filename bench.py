@@ -297,7 +297,7 @@ NCU_TRAFFIC = {
     "note_dw": "wg_tc_kernel alone (mean of fc1, fc2): dY 77.5 MB + dense scratch 19.4 MB read once; the decompress kernel "
                "before it moves another 32.2 MB through DRAM on fc2 (13.8 read, 18.4 written, the rest of its 77.5 MB "
                "output stays in L2 for the GEMM)",
-    "fused_compress_kernel_fc2": 78.481408e6 + 4.761088e6,
+    "fused_compress_kernel_fc2": 78.998016e6 + 3.350784e6,
 }
 
 
