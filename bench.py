@@ -6,6 +6,15 @@ tokens, gamma = 0.9): min-k compression of the fc1 and fc2 inputs, then both wei
 from the compressed caches.  One JSON line is printed by rank 0.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py --only OP:CASE[:GAMMA] [--reps R] [--queued] [--format bitmask|index32]
+
+The first form times exactly K steps (CUDA events on the stream the library is given), then the
+same step for at least a second (clocks under sustained load), the step from host buffers, and,
+on one GPU, the other named workloads (fp32 single Linear, ResNet-50 stage-1 convolutions,
+ViTDet-B linears at three drop ratios, the whole ViT-B/16 training step).
+The second form runs one entry point on one named workload a few times and prints each time:
+it is what the profiler command lines under profiles/ run.  OP is compress, compress_random,
+decompress, weight_grad or conv_weight_grad.
 
 N > 1 is launched with torch.distributed.run, one rank per GPU; the path has no exchange step,
 so ranks are independent replicas (weak scaling) and NCCL only carries the barrier and the
@@ -35,6 +44,9 @@ LAYERS = (di.VITB_FC1, di.VITB_FC2)
 WORKLOAD = "vitb16_mlp_fc1_fc2_batch64_gamma0.9"
 METRIC = "step samples/s (DropIT hot path: min-k compress + sparse-cache dW)"
 N_INPUT_SETS = 3   # distinct input batches rotated between steps; one batch is 194 MB (> 126 MB of L2)
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # datasheet figures, for context beside the measured ones
+CASES = {c.name: c for c in (di.SINGLE_LINEAR_F32, di.VITB_FC1, di.VITB_FC2, di.R50_CONV1X1, di.R50_CONV3X3,
+                             di.VITDET_QKV, di.VITDET_FC1, di.VITDET_FC2)}
 
 
 def measured_peaks():
@@ -74,47 +86,85 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
-    def stop(self, t0: float, t1: float):
+    def window(self, t0: float, t1: float):
+        """Median SM clock, maximum clock and throttle reasons seen between two wall-clock times."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.12)
-        self.proc.terminate()
         rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.1] or [l for (_, l) in self.lines]
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             f = [c.strip() for c in r.split(",")]
             try:
                 sm.append(float(f[0]))
                 mx.append(float(f[1]))
+                pw.append(float(f[2]))
             except (ValueError, IndexError):
                 continue
             for nm, val in zip(names, f[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(nm)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+    def stop(self):
+        if self.proc is not None:
+            time.sleep(0.12)
+            self.proc.terminate()
 
 
 # ------------------------------------------------------------------------------------------
-# the product arm
+# byte and flop counts of the method (what the rooflines divide)
 # ------------------------------------------------------------------------------------------
+def _elem_bytes(case) -> int:
+    return 2 if case.dtype == "bf16" else 4
+
+
 def algorithmic_bytes_compress(case) -> float:
-    """Radix select sees the tensor before and after the threshold is known: 2 reads of X, one write of
-    the mask, the retained values and the seek table."""
+    """Radix select sees the tensor before and after the threshold is known (bf16: 2 reads of X; fp32 keys take
+    three digit passes), and writes the mask, the retained values and the seek table."""
     import paper_2202_13808_b200 as dropit
-    n = case.n
+    n, es = case.n, _elem_bytes(case)
     k = dropit.dropit_keep_count(n, case.gamma)
-    return 2 * n * 2 + n / 8 + k * 2 + 4 * ((n + 127) // 128)
+    passes = 2 if es == 2 else 3
+    return passes * n * es + n / 8 + k * es + 4 * ((n + 127) // 128)
 
 
 def compulsory_bytes_compress(case) -> float:
     """One read of X plus the outputs: what any method has to move."""
-    return algorithmic_bytes_compress(case) - case.n * 2
+    import paper_2202_13808_b200 as dropit
+    n, es = case.n, _elem_bytes(case)
+    k = dropit.dropit_keep_count(n, case.gamma)
+    return n * es + n / 8 + k * es + 4 * ((n + 127) // 128)
+
+
+def algorithmic_bytes_dw(case) -> float:
+    """dY once, the compressed cache once, dW once."""
+    import paper_2202_13808_b200 as dropit
+    n, es = case.n, _elem_bytes(case)
+    k = dropit.dropit_keep_count(n, case.gamma)
+    cache = k * es + n / 8 + 4 * ((n + 127) // 128)
+    if isinstance(case, di.LinearCase):
+        return case.M * case.Cz * es + cache + case.Cz * case.Ca * 4
+    return case.B * case.Cz * case.Ho * case.Wo * es + cache + case.Cz * case.Ca * case.R * case.S * 4
 
 
 def dense_flops(case) -> float:
-    return 2.0 * case.M * case.Ca * case.Cz
+    """Flops of the zero-filled dense product the method prescribes (Eq. 4-6)."""
+    if isinstance(case, di.LinearCase):
+        return 2.0 * case.M * case.Ca * case.Cz
+    return 2.0 * case.B * case.Ho * case.Wo * case.Cz * case.Ca * case.R * case.S
+
+
+def fractions(achieved: float, kind: str, peaks) -> dict:
+    """The achieved rate against the measured burst peak, the measured sustained peak (tensor only) and the
+    datasheet figure."""
+    if kind == "tensor":
+        out = {"frac": achieved / peaks["bf16_tflops"], "frac_of_nominal": achieved / NOMINAL["bf16_tflops"]}
+        if peaks.get("bf16_tflops_sustained"):
+            out["frac_of_sustained"] = achieved / peaks["bf16_tflops_sustained"]
+        return out
+    return {"frac": achieved / peaks["hbm_gbs"], "frac_of_nominal": achieved / NOMINAL["hbm_gbs"]}
 
 
 def max_over_ranks(ms: float, world: int, device) -> float:
@@ -131,6 +181,145 @@ def whole_job_value(world: int, steps: int, ms: float) -> float:
     return world * BATCH_IMAGES * steps / (ms / 1e3)
 
 
+# ------------------------------------------------------------------------------------------
+# one entry point on one workload (also what --only runs)
+# ------------------------------------------------------------------------------------------
+class OpRunner:
+    """Holds the device tensors of one (op, case) pair over `nsets` rotating input sets and calls the op."""
+
+    def __init__(self, op: str, case, device, fmt: str = "bitmask", nsets: int = 3):
+        import paper_2202_13808_b200 as dropit
+        self.dropit, self.op, self.case, self.fmt, self.nsets, self.dev = dropit, op, case, fmt, nsets, device
+        need_dy = op in ("weight_grad", "conv_weight_grad")
+        self.xs = [di.make_x(case, b).to(device) for b in range(nsets)]
+        self.dys = [di.make_dy(case, b).to(device) for b in range(nsets)] if need_dy else None
+        self.caches = [dropit.dropit_compress(x, case.gamma, fmt) for x in self.xs]
+        if op not in ("compress", "compress_random"):
+            self.xs = None   # the dense inputs are not needed any more
+
+    def __call__(self, i: int):
+        d, c, b = self.dropit, self.case, i % self.nsets
+        if self.op == "compress":
+            self.caches[b] = d.dropit_compress(self.xs[b], c.gamma, self.fmt)
+        elif self.op == "compress_random":
+            self.caches[b] = d.dropit_compress_random(self.xs[b], c.gamma, i, self.fmt)
+        elif self.op == "decompress":
+            d.dropit_decompress(self.caches[b])
+        elif self.op == "weight_grad":
+            d.dropit_weight_grad(self.dys[b], self.caches[b])
+        elif self.op == "conv_weight_grad":
+            d.dropit_conv_weight_grad(self.dys[b], self.caches[b], (c.R, c.S), c.stride, c.pad)
+        else:
+            raise ValueError(self.op)
+
+    def queued_us(self, reps: int) -> float:
+        """Mean time of `reps` back-to-back calls over the rotating input sets (no host sync in between)."""
+        stream = torch.cuda.current_stream(self.dev)
+        for i in range(3):
+            self(i)
+        torch.cuda.synchronize(self.dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(reps):
+            self(i)
+        e1.record(stream)
+        torch.cuda.synchronize(self.dev)
+        return e0.elapsed_time(e1) / reps * 1e3
+
+
+def run_only(args, device):
+    parts = args.only.split(":")
+    op, case = parts[0], CASES[parts[1]]
+    if len(parts) > 2:
+        case = di.with_gamma(case, float(parts[2]))
+    import paper_2202_13808_b200 as dropit
+    run = OpRunner(op, case, device, args.format, 3 if args.queued else 1)
+    if args.queued:
+        us = run.queued_us(args.reps)
+        by = algorithmic_bytes_compress(case) if op.startswith("compress") else 0.0
+        fl = dense_flops(case) if op.endswith("weight_grad") else 0.0
+        rate = "%.0f GB/s algorithmic" % (by / us / 1e3) if by else ("%.0f TFLOP/s" % (fl / us / 1e6) if fl else "")
+        print("%s %s gamma=%g %s: %.1f us per call over %d queued calls %s"
+              % (op, case.name, case.gamma, args.format, us, args.reps, rate))
+    else:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        for r in range(args.reps):
+            flush.zero_()
+            torch.cuda.synchronize(device)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            run(r)
+            e1.record()
+            torch.cuda.synchronize(device)
+            print("%s %s gamma=%g rep %d: %.4f ms" % (op, case.name, case.gamma, r, e0.elapsed_time(e1)))
+    dropit.check_device_status(device)
+
+
+# ------------------------------------------------------------------------------------------
+# the other named workloads (one GPU only): per-call times and their rooflines
+# ------------------------------------------------------------------------------------------
+def other_workloads(device, peaks, reps: int = 20):
+    import paper_2202_13808_b200 as dropit
+    out = {}
+
+    def entry(case, op, us, launches):
+        e = {"us_per_call": us, "launches_per_call": launches}
+        if op == "compress":
+            a, c = algorithmic_bytes_compress(case), compulsory_bytes_compress(case)
+            e.update({"algorithmic_gbs": a / us / 1e3, "compulsory_gbs": c / us / 1e3})
+            e.update({"frac_" + k: v for k, v in (("algorithmic", a / us / 1e3 / peaks["hbm_gbs"]),
+                                                  ("compulsory", c / us / 1e3 / peaks["hbm_gbs"]))})
+        else:
+            fl, by = dense_flops(case), algorithmic_bytes_dw(case)
+            e.update({"tflops": fl / us / 1e6, "frac_of_bf16_peak": fl / us / 1e6 / peaks["bf16_tflops"],
+                      "algorithmic_gbs": by / us / 1e3, "frac_of_hbm_peak": by / us / 1e3 / peaks["hbm_gbs"]})
+        return e
+
+    def timed(case, op):
+        run = OpRunner(op, case, device, "bitmask", 3)
+        l0 = dropit.dropit_launch_count()
+        us = run.queued_us(reps)
+        launches = (dropit.dropit_launch_count() - l0) / (reps + 3)
+        del run
+        torch.cuda.empty_cache()
+        return entry(case, op, us, launches)
+
+    # configuration 1: latency-bound, no roofline claim
+    c1 = di.SINGLE_LINEAR_F32
+    out["single_linear_f32"] = {"compress": timed(c1, "compress"), "weight_grad": timed(c1, "weight_grad"),
+                                "note": "0.8 MB tensor: launch latency; no roofline claim"}
+    # configuration 3: the 1x1 convolution is bound by HBM (6.6 GFLOP on 54 MB), the 3x3 by the tensor cores
+    out["r50_conv1x1"] = {"compress": timed(di.R50_CONV1X1, "compress"),
+                          "conv_weight_grad": timed(di.R50_CONV1X1, "conv_weight_grad"), "bound": "hbm"}
+    out["r50_conv3x3"] = {"compress": timed(di.R50_CONV3X3, "compress"),
+                          "conv_weight_grad": timed(di.R50_CONV3X3, "conv_weight_grad"), "bound": "tensor"}
+    # configuration 4: ViTDet-B linears at three drop ratios
+    for base in (di.VITDET_QKV, di.VITDET_FC1, di.VITDET_FC2):
+        for g in (0.5, 0.8, 0.9):
+            case = di.with_gamma(base, g)
+            out["%s_g%g" % (base.name, g)] = {"compress": timed(case, "compress"), "weight_grad": timed(case, "weight_grad")}
+    return out
+
+
+def vit_step(device, batch: int = 64, gamma: float = 0.9, steps: int = 5):
+    """Configuration 5: the whole ViT-B/16 training step, stock layers against DropIT on every Linear."""
+    from paper_2202_13808_b200 import vit
+    res = {}
+    for name, g in (("dense", None), ("dropit", gamma)):
+        model = vit.build_vit_b16(g, device=device)
+        sps, peak, loss = vit.train_steps(model, batch, steps)
+        res[name] = {"samples_per_s": sps, "peak_step_bytes": peak, "loss": loss}
+        del model
+        torch.cuda.empty_cache()
+    res["speed_ratio"] = res["dropit"]["samples_per_s"] / res["dense"]["samples_per_s"]
+    res["peak_ratio"] = res["dropit"]["peak_step_bytes"] / max(res["dense"]["peak_step_bytes"], 1)
+    res["config"] = {"model": "ViT-B/16", "depth": 12, "batch": batch, "gamma": gamma, "dtype": "bf16", "steps": steps}
+    return res
+
+
+# ------------------------------------------------------------------------------------------
+# the product arm
+# ------------------------------------------------------------------------------------------
 def run_ours(args, rank, world, device):
     import paper_2202_13808_b200 as dropit
 
@@ -140,7 +329,7 @@ def run_ours(args, rank, world, device):
     dws = [torch.empty((c.Cz, c.Ca), dtype=torch.float32, device=device) for c in LAYERS]
     ws_c = [torch.empty(dropit.dropit_cache_sizes(c.n, c.gamma, dropit.BF16, dropit.FMT_BITMASK)[3], dtype=torch.uint8,
                         device=device) for c in LAYERS]
-    ws_g = [torch.empty(dropit.dropit_weight_grad_workspace(c.M, c.Ca, c.Cz, dropit.BF16, dropit.FMT_BITMASK),
+    ws_g = [torch.empty(dropit.dropit_weight_grad_workspace(c.M, c.Ca, c.Cz, dropit.BF16, dropit.FMT_BITMASK, device),
                         dtype=torch.uint8, device=device) for c in LAYERS]
     stream = torch.cuda.current_stream(device)
 
@@ -167,7 +356,7 @@ def run_ours(args, rank, world, device):
             torch.distributed.barrier()
         torch.cuda.synchronize(device)
 
-    # per-call events: [layer][0..2] per step
+    # ---- exactly K steps, with per-call events: [layer][0..2] per step ----
     evs = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in LAYERS] for _ in range(args.steps)]
     sampler = ClockSampler(device.index or 0)
     if rank == 0:
@@ -184,31 +373,36 @@ def run_ours(args, rank, world, device):
     barrier()
     t1 = time.time()
     launches = dropit.dropit_launch_count() - launches0
-    clocks = sampler.stop(t0, t1) if rank == 0 else None
     dropit.check_device_status(device)
     ms = max_over_ranks(e0.elapsed_time(e1), world, device)
-
     comp_ms = [statistics.mean(evs[i][li][0].elapsed_time(evs[i][li][1]) for i in range(args.steps)) for li in range(2)]
     dw_ms = [statistics.mean(evs[i][li][1].elapsed_time(evs[i][li][2]) for i in range(args.steps)) for li in range(2)]
 
-    # ---- the decompress launch of a dW call on its own (same caches, rotating), to split the call's time ----
-    caches = [[dropit.dropit_compress(sets[b][li][0], c.gamma, "bitmask", workspace=ws_c[li]) for li, c in enumerate(LAYERS)]
-              for b in range(N_INPUT_SETS)]
-    dense = [torch.empty(c.n, dtype=torch.bfloat16, device=device) for c in LAYERS]
-    dec_ms = []
-    for li in range(len(LAYERS)):
-        for i in range(6):
-            dropit.dropit_decompress(caches[i % N_INPUT_SETS][li], out=dense[li])
-        barrier()
-        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = 30
-        d0.record(stream)
-        for i in range(reps):
-            dropit.dropit_decompress(caches[i % N_INPUT_SETS][li], out=dense[li])
-        d1.record(stream)
-        barrier()
-        dec_ms.append(d0.elapsed_time(d1) / reps)
-    del caches, dense
+    # ---- the same step for at least a second: what a training loop sees once the clocks have settled ----
+    est = max(ms / args.steps, 1e-3)
+    n_sus = int(min(max(1000.0 / est, args.steps), 20000))
+    barrier()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ts0 = time.time()
+    s0.record(stream)
+    for i in range(n_sus):
+        step(i)
+    s1.record(stream)
+    barrier()
+    ts1 = time.time()
+    sus_ms = max_over_ranks(s0.elapsed_time(s1), world, device)
+    # per-call times under sustained load (events in a short second loop of 50 steps right behind it)
+    evs2 = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in LAYERS] for _ in range(50)]
+    for i in range(50):
+        step(i, evs2[i])
+    barrier()
+    sus_comp = [statistics.mean(e[li][0].elapsed_time(e[li][1]) for e in evs2) for li in range(2)]
+    sus_dw = [statistics.mean(e[li][1].elapsed_time(e[li][2]) for e in evs2) for li in range(2)]
+    clocks = sus_clocks = None
+    if rank == 0:
+        clocks = sampler.window(t0, t1)
+        sus_clocks = sampler.window(ts0, ts1)
+    dropit.check_device_status(device)
 
     # ---- end to end through the public API with host buffers ----
     host_in = [(di.make_x(c, 0).pin_memory(), di.make_dy(c, 0).pin_memory()) for c in LAYERS]
@@ -236,18 +430,40 @@ def run_ours(args, rank, world, device):
     f1.record(stream)
     barrier()
     e2e_ms = max_over_ranks(f0.elapsed_time(f1), world, device)
+    del sets, host_in, dev_in
+    torch.cuda.empty_cache()
 
     if rank != 0:
         return None
     peaks = measured_peaks()
     ms_per_step = ms / args.steps
     value = whole_job_value(world, args.steps, ms)
-    # dominant kernel: the fc weight-gradient GEMM (both layers have the same flop count)
+    # dominant kernel: the fc weight gradient (both layers have the same flop count); one launch per call
     F = dense_flops(LAYERS[0])
     dw_avg_ms = statistics.mean(dw_ms)
     tfl = F / (dw_avg_ms * 1e-3) / 1e12
-    comp_bytes = [algorithmic_bytes_compress(c) for c in LAYERS]
-    comp_gbs = [b / (t * 1e-3) / 1e9 for b, t in zip(comp_bytes, comp_ms)]
+    comp_a = [algorithmic_bytes_compress(c) for c in LAYERS]
+    comp_c = [compulsory_bytes_compress(c) for c in LAYERS]
+    comp_gbs = [b / (t * 1e-3) / 1e9 for b, t in zip(comp_a, comp_ms)]
+    comp_cgbs = [b / (t * 1e-3) / 1e9 for b, t in zip(comp_c, comp_ms)]
+    tr_dw, tr_c = NCU_TRAFFIC["weight_grad_kernel"], NCU_TRAFFIC["fused_compress_kernel_fc2"]
+    roof = {"kernel": "dropit_weight_grad (one launch: cache expanded into tensor memory in front of tcgen05.mma)",
+            "bound": "tensor", "achieved": tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "traffic": tr_dw, "peak_source": peaks["source"] + " burst", "flops_per_launch": F, "avg_ms": dw_avg_ms,
+            "per_layer_tflops": {"fc1": F / (dw_ms[0] * 1e-3) / 1e12, "fc2": F / (dw_ms[1] * 1e-3) / 1e12},
+            "algorithmic_bytes_per_launch": statistics.mean(algorithmic_bytes_dw(c) for c in LAYERS)}
+    roof.update(fractions(tfl, "tensor", peaks))
+    roof_c = {"kernel": "dropit_compress (one launch: sample, band histogram, threshold, ordered compaction)",
+              "bound": "hbm", "layer": LAYERS[1].name, "achieved": comp_gbs[1], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+              "bytes_per_call": comp_a[1], "avg_ms": comp_ms[1], "traffic": tr_c, "peak_source": peaks["source"],
+              "achieved_is": "algorithmic bytes (two reads of X + outputs) / time; the second read of this 77.5 MB "
+                             "tensor is served by L2, so the bytes that cross HBM are the compulsory ones",
+              "compulsory_gbs": comp_cgbs[1], "compulsory_frac": comp_cgbs[1] / peaks["hbm_gbs"],
+              "dram_gbs": tr_c / (comp_ms[1] * 1e-3) / 1e9 if tr_c else None,
+              "other_layer": {"layer": LAYERS[0].name, "achieved": comp_gbs[0], "frac": comp_gbs[0] / peaks["hbm_gbs"],
+                              "compulsory_gbs": comp_cgbs[0], "avg_ms": comp_ms[0],
+                              "note": "19.4 MB: fits L2, dominated by the kernel's fixed steps"}}
+    roof_c.update(fractions(comp_gbs[1], "hbm", peaks))
     out = {
         "metric": METRIC, "value": value, "unit": "samples/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -255,49 +471,37 @@ def run_ours(args, rank, world, device):
         "config": {"workload": WORKLOAD, "layers": [c.name for c in LAYERS], "tokens": LAYERS[0].M, "gamma": 0.9,
                    "format": "bitmask", "l2": "inputs rotate over %d batches of 194 MB each (> L2)" % N_INPUT_SETS,
                    "parallelism": "replicas x%d" % world},
-        "roofline": {"kernel": "dropit_weight_grad (tcgen05 GEMM incl. its decompress)", "bound": "tensor",
-                     "achieved": tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tfl / peaks["bf16_tflops"],
-                     "traffic": NCU_TRAFFIC["wg_tc_kernel"], "traffic_note": NCU_TRAFFIC["note_dw"],
-                     "peak_source": peaks["source"] + " burst", "flops_per_launch": F, "avg_ms": dw_avg_ms},
-        "roofline_compress": {"kernel": "dropit_compress (histogram + compaction)", "bound": "hbm",
-                              "achieved": comp_gbs[1], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                              "frac": comp_gbs[1] / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC["fused_compress_kernel_fc2"],
-                              "peak_source": peaks["source"], "bytes_per_call": comp_bytes[1], "avg_ms": comp_ms[1],
-                              "compulsory_gbs": compulsory_bytes_compress(LAYERS[1]) / (comp_ms[1] * 1e-3) / 1e9,
-                              "dram_gbs": (NCU_TRAFFIC["fused_compress_kernel_fc2"] / (comp_ms[1] * 1e-3) / 1e9
-                                           if NCU_TRAFFIC["fused_compress_kernel_fc2"] else None),
-                              "layer": LAYERS[1].name,
-                              "other_layer": {"layer": LAYERS[0].name, "achieved": comp_gbs[0],
-                                              "frac": comp_gbs[0] / peaks["hbm_gbs"], "avg_ms": comp_ms[0]}},
-        "roofline_gemm_kernel": {"kernel": "wg_tc_kernel alone, estimated on fc2: the dW call minus its decompress launch, which "
-                                           "was timed separately on the same caches (the two launches overlap by the GEMM's "
-                                           "set-up; fc1's decompress is too short to time from the host; the launch-list "
-                                           "shares under profiles/ agree with the estimate)",
-                                 "bound": "tensor", "unit": "TFLOP/s", "peak": peaks["bf16_tflops"],
-                                 "achieved": F / ((dw_ms[1] - dec_ms[1]) * 1e-3) / 1e12,
-                                 "frac": F / ((dw_ms[1] - dec_ms[1]) * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                                 "decompress_ms": {"fc1_host_bound": dec_ms[0], "fc2": dec_ms[1]}},
+        "roofline": roof,
+        "roofline_compress": roof_c,
         "per_call_ms": {"compress_fc1": comp_ms[0], "compress_fc2": comp_ms[1], "dw_fc1": dw_ms[0], "dw_fc2": dw_ms[1]},
-        "dw_tflops": {"fc1": F / (dw_ms[0] * 1e-3) / 1e12, "fc2": F / (dw_ms[1] * 1e-3) / 1e12},
+        "sustained": {"steps": n_sus, "seconds": sus_ms / 1e3, "ms_per_step": sus_ms / n_sus,
+                      "value": whole_job_value(world, n_sus, sus_ms), "clocks": sus_clocks,
+                      "per_call_ms": {"compress_fc1": sus_comp[0], "compress_fc2": sus_comp[1], "dw_fc1": sus_dw[0],
+                                      "dw_fc2": sus_dw[1]},
+                      "dw_tflops": F / (statistics.mean(sus_dw) * 1e-3) / 1e12,
+                      "dw_frac_of_sustained_peak": (F / (statistics.mean(sus_dw) * 1e-3) / 1e12 /
+                                                    peaks["bf16_tflops_sustained"]) if peaks.get("bf16_tflops_sustained") else None,
+                      "compress_fc2_gbs": comp_a[1] / (sus_comp[1] * 1e-3) / 1e9},
         "e2e": {"value": whole_job_value(world, e2e_steps, e2e_ms), "unit": "samples/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if world == 1 and not args.skip_extras:
+        out["workloads"] = other_workloads(device, peaks)
+        out["vit_b16_step"] = vit_step(device)
+        dropit.check_device_status(device)
+    sampler.stop()
     if world == 1:
         out["cpu_baseline"] = cpu_baseline_sample()
     return out
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (weight_grad_gemm_wg_tc_kernel_vitb_fc1/fc2.txt, compress_fused_vitb_fc2.txt).  Set an entry to None
-# when its kernel changes, until the counters have been taken again.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/.
+# An entry is None from the moment its kernel changes until the counters have been taken again.
 NCU_TRAFFIC = {
-    "wg_tc_kernel": 0.5 * ((96.877056e6 + 4.115456e6) + (96.871424e6 + 4.160256e6)),
-    "note_dw": "wg_tc_kernel alone (mean of fc1, fc2): dY 77.5 MB + dense scratch 19.4 MB read once; the decompress kernel "
-               "before it moves another 32.2 MB through DRAM on fc2 (13.8 read, 18.4 written, the rest of its 77.5 MB "
-               "output stays in L2 for the GEMM)",
-    "fused_compress_kernel_fc2": 78.998016e6 + 3.350784e6,
+    "weight_grad_kernel": None,
+    "fused_compress_kernel_fc2": None,
 }
 
 
@@ -368,6 +572,13 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--skip-extras", action="store_true", help="leave out the other workloads and the ViT-B/16 step")
+    ap.add_argument("--only", default=None, help="OP:CASE[:GAMMA]: run one entry point on one workload, for profilers")
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--queued", action="store_true",
+                    help="with --only: time all repetitions as one region over 3 rotating input sets (no host sync "
+                         "between calls); default: one flushed, synchronised call per line")
+    ap.add_argument("--format", default="bitmask", choices=["bitmask", "index32"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -385,6 +596,9 @@ def main():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
+    if args.only:
+        run_only(args, device)
+        return 0
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         torch.distributed.init_process_group("nccl", device_id=device)

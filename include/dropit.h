@@ -197,12 +197,14 @@ dropit_status dropit_weight_grad(const void* dy, const void* values, const void*
 
 /*
  * Same result as dropit_weight_grad (Eq. 6), computed WITHOUT inflating the cache to a dense
- * scratch tensor: mask, seek table and packed values are prefetched into shared memory and the
- * R(a-hat) tiles (Sec. 3.2) are built there, right in front of the tensor cores.  Needs
- * dtype = DROPIT_BF16, format = DROPIT_FMT_BITMASK, Ca a multiple of 128 and Cz a multiple of 8;
- * anything else returns DROPIT_ERR_UNSUPPORTED.  Same arguments and workspace size as
- * dropit_weight_grad, of which it uses less (no dense scratch is touched).  On B200 it is the
- * slower of the two variants; dropit_weight_grad never takes it on its own.
+ * scratch tensor: R(a-hat) (Sec. 3.2: recovery is a temporary) is rebuilt, 32 tokens x 32 channels
+ * at a time, straight from mask words, seek-table entries and packed values, and stored into
+ * tensor memory, where the tensor cores read it as an MMA operand.  One kernel launch, and the
+ * workspace is not touched (it may be NULL / 0 bytes).  Needs dtype = DROPIT_BF16,
+ * format = DROPIT_FMT_BITMASK, Ca a multiple of 128 and Cz a multiple of 8; anything else
+ * returns DROPIT_ERR_UNSUPPORTED.  On B200 it is the slower of the two variants (the expansion,
+ * not the tensor cores, sets its pace), so dropit_weight_grad does not take it on its own; it
+ * is for callers that cannot spare the n * 2 bytes of scratch.  Same summation-order guarantee.
  */
 dropit_status dropit_weight_grad_fused(const void* dy, const void* values, const void* meta, const uint32_t* offsets,
                                        int64_t M, int64_t Ca, int64_t Cz, int64_t k, dropit_dtype dtype,

@@ -198,12 +198,25 @@ def dropit_decompress(cache: DropITCache, out: Optional[torch.Tensor] = None) ->
     return out
 
 
+def _device_index(device) -> int:
+    if device is None:
+        return torch.cuda.current_device()
+    device = torch.device(device)
+    return torch.cuda.current_device() if device.index is None else device.index
+
+
 @functools.lru_cache(maxsize=4096)
-def dropit_weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int) -> int:
+def _weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int, dev_index: int) -> int:
     out = ctypes.c_size_t(0)
-    _check(_lib.load().dropit_weight_grad_workspace(M, Ca, Cz, dtype, fmt, ctypes.byref(out)),
-           "dropit_weight_grad_workspace")
+    with _on_device(torch.device("cuda", dev_index)):
+        code = _lib.load().dropit_weight_grad_workspace(M, Ca, Cz, dtype, fmt, ctypes.byref(out))
+    _check(code, "dropit_weight_grad_workspace")
     return int(out.value)
+
+
+def dropit_weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int, device=None) -> int:
+    """Scratch bytes of dropit_weight_grad on `device` (the plan depends on the device's SM count)."""
+    return _weight_grad_workspace(int(M), int(Ca), int(Cz), int(dtype), int(fmt), _device_index(device))
 
 
 def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch.Tensor] = None,
@@ -227,7 +240,7 @@ def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch
         if accumulate:
             raise ValueError("accumulate=True needs out")
         out = torch.empty((Cz, Ca), dtype=torch.float32, device=dev)
-    wb = dropit_weight_grad_workspace(M, Ca, Cz, dt, cache.fmt)
+    wb = dropit_weight_grad_workspace(M, Ca, Cz, dt, cache.fmt, dev)
     if workspace is None or workspace.numel() < wb:
         workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
     with _on_device(dev):
@@ -240,11 +253,18 @@ def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch
 
 
 @functools.lru_cache(maxsize=4096)
-def dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype: int, fmt: int) -> int:
+def _conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype: int, fmt: int, dev_index: int) -> int:
     out = ctypes.c_size_t(0)
-    _check(_lib.load().dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype, fmt,
-                                                         ctypes.byref(out)), "dropit_conv_weight_grad_workspace")
+    with _on_device(torch.device("cuda", dev_index)):
+        code = _lib.load().dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype, fmt,
+                                                             ctypes.byref(out))
+    _check(code, "dropit_conv_weight_grad_workspace")
     return int(out.value)
+
+
+def dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dtype: int, fmt: int, device=None) -> int:
+    """Scratch bytes of dropit_conv_weight_grad on `device` (the split count depends on its SM count)."""
+    return _conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, int(dtype), int(fmt), _device_index(device))
 
 
 def dropit_conv_weight_grad(dy: torch.Tensor, cache: DropITCache, kernel_size: Tuple[int, int], stride: int = 1,
@@ -264,7 +284,7 @@ def dropit_conv_weight_grad(dy: torch.Tensor, cache: DropITCache, kernel_size: T
         if accumulate:
             raise ValueError("accumulate=True needs out")
         out = torch.empty((Cz, Ca, R, S), dtype=torch.float32, device=dev)
-    wb = dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dt, cache.fmt)
+    wb = dropit_conv_weight_grad_workspace(B, Ca, H, W, Cz, R, S, stride, pad, dt, cache.fmt, dev)
     if workspace is None or workspace.numel() < wb:
         workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
     with _on_device(dev):

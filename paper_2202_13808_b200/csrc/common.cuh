@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "dropit.h"
 
 namespace dropit {
@@ -74,6 +76,36 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // Number of SMs of the current device (cached per device id).
 int sm_count();
 
+// Index of the current device, or -1.
+inline int current_device() {
+    int dev = 0;
+    return (cudaGetDevice(&dev) == cudaSuccess && dev >= 0) ? dev : -1;
+}
+
+// Kernel attributes (dynamic shared memory size, ...) belong to a device, not to the process: a call
+// site keeps one of these and sets its attributes the first time it runs on each device.
+struct PerDeviceOnce {
+    std::atomic<bool> done[64];
+    bool needed() const {
+        const int dev = current_device();
+        return dev < 0 || dev >= 64 || !done[dev].load(std::memory_order_acquire);
+    }
+    void mark() {
+        const int dev = current_device();
+        if (dev >= 0 && dev < 64) done[dev].store(true, std::memory_order_release);
+    }
+};
+
+// A number that no earlier call of this process has used (and that another process is unlikely to
+// have left in recycled memory): device-side barriers and ready flags that live in scratch memory
+// nobody cleared tell this call's marks from stale ones by it.
+uint32_t next_epoch();
+
+// Polls that a bounded device-side wait makes before it gives up.  The defaults are far above any real
+// wait; the environment variable DROPIT_TEST_SPIN_LIMIT (read at every call, tests only) overrides them
+// so that the give-up paths can be exercised without hanging anything.
+uint32_t spin_limit(uint32_t default_limit);
+
 // Host-side shape of the compress workspace.
 struct CompressPlan {
     int64_t n;
@@ -88,11 +120,11 @@ CompressPlan make_compress_plan(int64_t n, int64_t k, dropit_dtype dtype);
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
 // Kernel launches enqueued by this library since it was loaded (diagnostic counter).
-extern unsigned long long g_launch_count;
+extern std::atomic<unsigned long long> g_launch_count;
 
 // Call once after every kernel launch.
 inline dropit_status check_launch() {
-    ++g_launch_count;
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? DROPIT_OK : DROPIT_ERR_CUDA;
 }
 

@@ -11,9 +11,30 @@
 //      retained elements before i is then  gt_before(i) + min(eq_before(i), q), so a single
 //      prefix sum over (gt, eq) counts places every value.  The prefix across tiles is a
 //      decoupled look-back over 64-bit tile descriptors with a bounded wait.
+#include <unistd.h>
+
+#include <chrono>
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace dropit {
+
+uint32_t next_epoch() {
+    static std::atomic<uint32_t> counter{[] {
+        const uint64_t t = (uint64_t)std::chrono::steady_clock::now().time_since_epoch().count();
+        uint64_t h = (t ^ ((uint64_t)getpid() << 32)) * 0x9E3779B97F4A7C15ull;
+        return (uint32_t)(h >> 32);
+    }()};
+    return counter.fetch_add(1u, std::memory_order_relaxed);
+}
+
+uint32_t spin_limit(uint32_t default_limit) {
+    const char* e = std::getenv("DROPIT_TEST_SPIN_LIMIT");
+    if (!e || !*e) return default_limit;
+    const long v = std::strtol(e, nullptr, 10);
+    return v > 0 ? (uint32_t)v : default_limit;
+}
 
 int sm_count() {
     static int cached[64] = {0};
@@ -447,11 +468,11 @@ static dropit_status launch_hist(const void* x, int64_t n, int64_t k, SelectStat
                                  cudaStream_t stream) {
     auto kern = hist_select_kernel<Tr, BITS, SHIFT, PASS, FIRST, LAST>;
     const size_t smem = (size_t)(1 << BITS) * 4;
-    static bool attr_set = false;   // per instantiation
-    if (!attr_set && smem > 48 * 1024) {
+    static PerDeviceOnce attr;   // per instantiation
+    if (smem > 48 * 1024 && attr.needed()) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return DROPIT_ERR_CUDA;
-        attr_set = true;
+        attr.mark();
     }
     const int64_t nvec = n / Tr::kVecElems;
     int64_t blocks = (nvec + (int64_t)kHistThreads * 4 - 1) / ((int64_t)kHistThreads * 4);
@@ -472,11 +493,11 @@ static dropit_status launch_compact(const void* x, const CompressPlan& plan, Sel
     constexpr int A = 16 / Tr::kElemBytes;
     size_t smem = (size_t)(TILE_ELEMS + A) * Tr::kElemBytes;
     if (INDEX32) smem += (size_t)(TILE_ELEMS + 4) * 4;
-    static bool attr_set = false;
-    if (!attr_set && smem > 48 * 1024) {
+    static PerDeviceOnce attr;
+    if (smem > 48 * 1024 && attr.needed()) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return DROPIT_ERR_CUDA;
-        attr_set = true;
+        attr.mark();
     }
     kern<<<(unsigned)plan.n_tiles, kCompactThreads, smem, stream>>>(
         reinterpret_cast<const uint4*>(x), plan.n, st, desc, reinterpret_cast<typename Tr::elem_t*>(values),

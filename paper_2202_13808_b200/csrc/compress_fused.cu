@@ -21,10 +21,6 @@
 // full CTA histogram in shared memory, global histogram by atomics, then one extra counting read.
 // Nothing in the scratch has to be cleared before a call: the grid barrier counts arrivals under a
 // number unique to the call, everything else is written before it is read.
-#include <unistd.h>
-
-#include <atomic>
-#include <chrono>
 #include <type_traits>
 
 #include "common.cuh"
@@ -94,17 +90,6 @@ static FusedPlan make_fused_plan(int64_t n) {
 }
 
 size_t fused_compress_workspace_bytes(int64_t n) { return make_fused_plan(n).total_bytes; }
-
-// A number that no earlier call of this process has used (and that another process is unlikely to
-// have left in recycled memory): the grid barrier tells its own arrivals from stale ones by it.
-static uint32_t next_epoch() {
-    static std::atomic<uint32_t> counter{[] {
-        const uint64_t t = (uint64_t)std::chrono::steady_clock::now().time_since_epoch().count();
-        uint64_t h = (t ^ ((uint64_t)getpid() << 32)) * 0x9E3779B97F4A7C15ull;
-        return (uint32_t)(h >> 32);
-    }()};
-    return counter.fetch_add(1u, std::memory_order_relaxed);
-}
 
 __device__ __forceinline__ uint32_t ptx_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -302,7 +287,8 @@ __device__ __forceinline__ void barrier_open(unsigned long long* word, uint32_t 
         asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(word), "l"((unsigned long long)epoch << 32) : "memory");
     }
 }
-__device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t epoch, uint32_t target, int* s_ok) {
+__device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t epoch, uint32_t target, int* s_ok,
+                                             int spin_max) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
@@ -312,7 +298,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t 
         for (;;) {   // the word belongs to this call
             asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(word) : "memory");
             if ((uint32_t)(v >> 32) == epoch) break;
-            if (++spins > kBarrierSpinLimit) { ok = false; break; }
+            if (++spins > spin_max) { ok = false; break; }
             __nanosleep(32);
         }
         if (ok) {
@@ -321,7 +307,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t 
             for (;;) {
                 asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(word) : "memory");
                 if (v >= goal) break;
-                if (++spins > kBarrierSpinLimit) { ok = false; break; }
+                if (++spins > spin_max) { ok = false; break; }
                 __nanosleep(32);
             }
         }
@@ -446,7 +432,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long k, int blocks_per_warp, uint32_t epoch,
                       unsigned char* ws, size_t hist_off0, size_t hist_off1, size_t agg_off, size_t rows_off,
                       uint16_t* __restrict__ values, uint32_t* __restrict__ mask, int32_t* __restrict__ indices,
-                      uint32_t* __restrict__ offsets, int32_t* dev_status) {
+                      uint32_t* __restrict__ offsets, int32_t* dev_status, int spin_max) {
     // shared memory: [input ring, 128 KB | general path: full key histogram]
     //                [phase 3: per-warp value staging, 64 KB | sample step: 16-bit key histogram]
     //                [control block of phases 1-2]
@@ -637,7 +623,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             // grid barrier separates the clearing from the accumulation
             for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i <= width; i += gridDim.x * blockDim.x) ghist[i] = 0;
             barrier_target += gridDim.x;
-            if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok)) {
+            if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok, spin_max)) {
                 if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
                 return;
             }
@@ -648,7 +634,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             if (threadIdx.x == 0 && cta_hi) atomicAdd(&st->n_hi[attempt], (unsigned long long)cta_hi);
         }
         barrier_target += gridDim.x;
-        if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok)) {
+        if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok, spin_max)) {
             if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
             return;
         }
@@ -826,7 +812,7 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
             }
             if (threadIdx.x == 0) st_relaxed_u64(&agg[blockIdx.x], ((unsigned long long)ce << 32) | cg);
             barrier_target += gridDim.x;
-            if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok)) {
+            if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok, spin_max)) {
                 if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
                 return;
             }
@@ -987,12 +973,12 @@ dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool inde
     static_assert(kRingBytes >= (size_t)kKeySpace * 4, "the sample's and the general path's histogram live in the ring's memory");
     const size_t smem_mask = kRingBytes + kStageBytes + sizeof(FusedShared);
     const size_t smem_idx = smem_mask;   // indices are written from registers, not staged
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr;
+    if (attr.needed()) {
         if (cudaFuncSetAttribute(fused_compress_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_mask) != cudaSuccess ||
             cudaFuncSetAttribute(fused_compress_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_idx) != cudaSuccess)
             return DROPIT_ERR_CUDA;
-        attr_set = true;
+        attr.mark();
     }
     const uint4* xp = reinterpret_cast<const uint4*>(x);
     unsigned long long kk = (unsigned long long)k;
@@ -1002,7 +988,8 @@ dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool inde
     uint16_t* vals = reinterpret_cast<uint16_t*>(values);
     uint32_t* maskp = index32 ? nullptr : reinterpret_cast<uint32_t*>(meta);
     int32_t* idxp = index32 ? reinterpret_cast<int32_t*>(meta) : nullptr;
-    void* args[] = {&xp, &n, &kk, &bpw, &epoch, &ws, &h0, &h1, &ao, &ro, &vals, &maskp, &idxp, &offsets, &dev_status};
+    int spin_max = (int)spin_limit((uint32_t)kBarrierSpinLimit);
+    void* args[] = {&xp, &n, &kk, &bpw, &epoch, &ws, &h0, &h1, &ao, &ro, &vals, &maskp, &idxp, &offsets, &dev_status, &spin_max};
     const void* fn = index32 ? (const void*)fused_compress_kernel<true> : (const void*)fused_compress_kernel<false>;
     if (cudaLaunchCooperativeKernel(fn, dim3(plan.grid), dim3(kFusedThreads), args, index32 ? smem_idx : smem_mask,
                                     stream) != cudaSuccess) {

@@ -510,12 +510,12 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
     if (!make_map_nchw(&maps.dy, dy_gemm, B, Cz, pl.Ho, pl.Wop, pl.p.xb, pl.p.yb, pl.p.a_rows)) return DROPIT_ERR_CUDA;
     if (!make_map_taps(&maps.x, ws, B, Ca, pl.Hx, pl.Wp, pl.copies, pl.dense_stride, pl.p.bnc, pl.p.nv))
         return DROPIT_ERR_CUDA;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr;
+    if (attr.needed()) {
         if (cudaFuncSetAttribute(conv_wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kConvTcSmemBytes) != cudaSuccess)
             return DROPIT_ERR_CUDA;
-        attr_set = true;
+        attr.mark();
     }
     float* partial = reinterpret_cast<float*>(ws + pl.partial_off);
     dim3 grid(pl.tiles, pl.p.splits);

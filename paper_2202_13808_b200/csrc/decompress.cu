@@ -6,7 +6,7 @@
 
 namespace dropit {
 
-unsigned long long g_launch_count = 0;
+std::atomic<unsigned long long> g_launch_count{0};
 
 // A warp inflates 1024 consecutive elements (32 mask words, 8 chunks) per step: lane l owns word l, and the
 // lane's first value sits at the chunk's table entry plus the population of the chunk's earlier words.
@@ -288,7 +288,7 @@ extern "C" dropit_status dropit_decompress(const void* values, const void* meta,
 
 extern "C" int dropit_version(void) { return 100; }
 
-extern "C" uint64_t dropit_launch_count(void) { return g_launch_count; }
+extern "C" uint64_t dropit_launch_count(void) { return g_launch_count.load(std::memory_order_relaxed); }
 
 extern "C" const char* dropit_status_string(dropit_status s) {
     switch (s) {

@@ -5,14 +5,21 @@
 // operands, so for the tensor cores both operands are "MN-major": A = dY^T tile (128 output rows j),
 // B = R(a-hat) tile (256 output columns c), K = 64 tokens per pipeline stage.
 //
-// bf16: tcgen05.mma (kind::f16, fp32 accumulators in TMEM), operands staged in shared memory in the
-// 128-byte-swizzled canonical layout.  The bitmask cache is expanded inside the GEMM
-// (weight_grad_fused.cu).  This file holds the variant for the int32-index format and for channel
-// counts that are not a multiple of 128: the cache is first inflated to a dense scratch tensor and
-// both operands arrive by TMA; one warp issues TMA, one thread issues MMAs, four warps drain TMEM.
-// Small output matrices are split along n ("split-K"); each split stores its partial tile and the
-// last split to arrive adds the partials in split order, so the summation order is fixed.
-// fp32 (and shapes the TMA path cannot take): an FFMA kernel with 64x64 tiles.
+// bf16: tcgen05.mma (kind::f16, fp32 accumulators in TMEM).  Two kernels:
+//  * this file: the cache is first inflated to a dense scratch matrix by the decompression kernel (it mostly stays
+//    in L2), both operands arrive by TMA in the 128-byte-swizzled canonical layout; one warp issues TMA, one
+//    thread issues MMAs, four warps drain TMEM.  The GEMM is launched programmatically behind the decompression
+//    and sets itself up while that one drains.  This is the faster variant on every measured shape and what
+//    dropit_weight_grad takes.
+//  * weight_grad_tmem.cu (dropit_weight_grad_fused): no scratch; the cache is expanded into tensor memory in
+//    front of the MMAs.  One launch, no workspace, slower.
+// Small output matrices are split along n ("split-K").  2 or 4 splits of a tile form a thread-block cluster and
+// add up through distributed shared memory; other split counts store partial tiles and the last split to arrive
+// adds them in split order.  Either way the summation order is fixed.
+// fp32 (and channel counts that are not a multiple of 8): an FFMA kernel with 64x64 tiles on the dense scratch.
+#include <cstdlib>
+#include <cstring>
+
 #include "weight_grad_common.cuh"
 
 namespace dropit {
@@ -23,16 +30,14 @@ dropit_status decompress_dispatch(const void* values, const void* meta, const ui
 // ---------------------------------------------------------------------------------------------
 // Plan
 // ---------------------------------------------------------------------------------------------
-#ifndef DROPIT_FUSED_MIN_TOKENS
-#define DROPIT_FUSED_MIN_TOKENS (1ll << 40)   // never: the dense-scratch variant is faster on every measured shape so far
-#endif
-constexpr int64_t kFusedMinTokens = DROPIT_FUSED_MIN_TOKENS;   // see make_wg_plan
 constexpr int kStages = 4;
-constexpr int kTcThreads = 192;
+constexpr int kEpiSubs = 1;                            // epilogue warps per TMEM lane quarter (more of them did not shorten the epilogue)
+constexpr int kEpiWarps = 4 * kEpiSubs;
+constexpr int kTcThreads = 64 + 32 * kEpiWarps;        // TMA warp, MMA warp, epilogue warps (idle until the accumulator is final)
 
 struct WgPlan {
     bool tensor_core;
-    bool fused;               // expand the bitmask cache inside the GEMM (no dense scratch)
+    bool fused;               // weight_grad_tmem.cu: the cache is expanded into tensor memory inside the GEMM (no dense scratch)
     bool cluster;             // the splits of a tile form a thread-block cluster and add up through shared memory
     int tiles_m, tiles_n, splits, kb_total, kb_per_split;
     size_t counters_off, counters_bytes;
@@ -41,18 +46,32 @@ struct WgPlan {
     size_t total_bytes;
 };
 
-static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format,
-                           bool force_fused = false) {
+// The kernel without a scratch: bitmask caches whose rows are whole 128-element chunks.
+static bool fused_supported(int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format) {
+    return dtype == DROPIT_BF16 && format == DROPIT_FMT_BITMASK && (Ca % DROPIT_CHUNK == 0) && (Cz % 8 == 0);
+}
+
+static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format, bool fused) {
     WgPlan p{};
     p.tensor_core = (dtype == DROPIT_BF16) && (Ca % 8 == 0) && (Cz % 8 == 0);
-    // The in-kernel cache expansion (weight_grad_fused.cu) is taken on request (dropit_weight_grad_fused)
-    // or above a token count; on B200 the dense-scratch variant has been faster on every measured shape.
-    const bool fused_ok = p.tensor_core && format == DROPIT_FMT_BITMASK && (Ca % DROPIT_CHUNK == 0);
-    p.fused = fused_ok && (force_fused || M >= kFusedMinTokens);
+    p.fused = fused && fused_supported(Ca, Cz, dtype, format);
     const size_t es = (dtype == DROPIT_BF16) ? 2 : 4;
+    if (p.fused) {
+        // tiles of 128 channels x 256 outputs; the splits of the token axis are the CTAs of a cluster (1, 2 or 4)
+        p.tiles_m = (int)(Ca / kBM);
+        p.tiles_n = (int)((Cz + kBN - 1) / kBN);
+        p.kb_total = (int)((M + kBK - 1) / kBK);
+        int want = sm_count() / (p.tiles_m * p.tiles_n);
+        want = want >= 4 ? 4 : (want >= 2 ? 2 : 1);
+        while (want > 1 && (p.kb_total + want - 1) / want * (want - 1) >= p.kb_total) want /= 2;   // every split owns >= 1 block
+        p.splits = want;
+        p.kb_per_split = (p.kb_total + want - 1) / want;
+        p.cluster = want > 1;
+        p.total_bytes = 256;
+        return p;
+    }
     if (p.tensor_core) {
-        const int tile_rows = p.fused ? kBM * kFusedAcc : kBM;
-        p.tiles_m = (int)((Cz + tile_rows - 1) / tile_rows);
+        p.tiles_m = (int)((Cz + kBM - 1) / kBM);
         p.tiles_n = (int)((Ca + kBN - 1) / kBN);
         p.kb_total = (int)((M + kBK - 1) / kBK);
         const int tiles = p.tiles_m * p.tiles_n;
@@ -61,7 +80,7 @@ static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype
         if (splits > p.kb_total) splits = p.kb_total;
         p.kb_per_split = (p.kb_total + splits - 1) / splits;
         p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;   // every split owns >= 1 block
-        p.cluster = !p.fused && (p.splits == 2 || p.splits == 4);
+        p.cluster = p.splits == 2 || p.splits == 4;
     } else {
         p.tiles_m = (int)((Cz + 63) / 64);
         p.tiles_n = (int)((Ca + 63) / 64);
@@ -70,7 +89,7 @@ static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype
     p.counters_off = 0;
     p.counters_bytes = align_up((size_t)p.tiles_m * p.tiles_n * 8, 256);   // per tile: tickets drawn, partial planes published
     p.dense_off = p.counters_off + p.counters_bytes;
-    p.dense_bytes = p.fused ? 0 : align_up((size_t)M * Ca * es, 256);
+    p.dense_bytes = align_up((size_t)M * Ca * es, 256);
     p.partial_off = p.dense_off + p.dense_bytes;
     p.partial_bytes = (p.splits > 1 && !p.cluster) ? align_up((size_t)p.splits * Cz * Ca * 4, 256) : 0;
     p.total_bytes = p.partial_off + p.partial_bytes;
@@ -112,7 +131,7 @@ bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t 
 // The same matrix seen as [cols / 64][rows][64]: one box {64, kBK, groups} brings `groups` adjacent 64-column
 // groups of kBK rows with a single copy, laid out group after group as the MN-major operand wants them.
 // Needs cols % 64 == 0 (a partial last group would read past the end of a row).
-static bool make_map_grouped_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int groups) {
+bool make_map_grouped_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int groups) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
@@ -138,8 +157,6 @@ struct TcSmem {
 constexpr int kEpiRowFloats = 36;                          // staging row pitch: 32 columns + 4 (bank spread, 16-byte rows)
 constexpr int kEpiWarpFloats = 32 * kEpiRowFloats;         // one warp's 32 x 32 chunk
 constexpr int kEpiSpinLimit = 1 << 20;
-// cluster exchange, receive area: (splits - 1) slots x 128 rows x (256 / splits + 4) floats; largest for 4 splits
-constexpr int kXchgMaxBytes = 3 * kBM * (kBN / 4 + 4) * 4;
 constexpr size_t kTcSmemBytes = 1024 + (size_t)kStages * (kAStageBytes + kBStageBytes) + sizeof(TcSmem);
 
 // Epilogue of one 128 x 256 accumulator tile, run by the four warps that own the TMEM lane quarters.
@@ -147,14 +164,14 @@ constexpr size_t kTcSmemBytes = 1024 + (size_t)kStages * (kAStageBytes + kBStage
 // 128-byte row segments.  A CTA that is not its tile's finisher stores the chunk into its split's
 // partial plane.  The finisher adds the planes in split order, taking its own term from the chunk, so
 // the sum does not depend on which split finishes last, and writes dW.
-__device__ __forceinline__ void epilogue_tile_staged(uint32_t tmem_base, float* stage, int g, int lane, int j0, int c0,
+__device__ __forceinline__ void epilogue_tile_staged(uint32_t tmem_base, float* stage, int g, int sub, int lane, int j0, int c0,
                                                      int Ca, int Cz, int split, int splits, bool finisher,
                                                      float* __restrict__ dw, int accumulate,
                                                      float* __restrict__ partial) {
     const size_t plane = (size_t)Cz * Ca;
     const int rr0 = lane >> 3, q = lane & 7;
 #pragma unroll 1
-    for (int ch = 0; ch < kBN / 32; ++ch) {
+    for (int ch = sub; ch < kBN / 32; ch += kEpiSubs) {    // the warps of a lane quarter take every kEpiSubs-th chunk
         const int col = c0 + ch * 32 + 4 * q;
         const bool col_ok = col < Ca;            // Ca is a multiple of 8
         size_t off[8];
@@ -224,44 +241,15 @@ __device__ __forceinline__ void epilogue_tile_staged(uint32_t tmem_base, float* 
     }
 }
 
-// Split reduction inside a thread-block cluster (2 or 4 splits of one tile are the CTAs of one cluster).
-// The tile's eight 32-column chunks are shared out among the CTAs (chunk ch belongs to CTA ch / (8 / splits)).
-// Every epilogue warp sends the chunks of its 32-row quarter that its CTA does not own from TMEM into the
-// owner's shared memory, and after a cluster barrier finishes the chunks its CTA owns: it adds the terms in
-// split order (its own from TMEM) and writes dW.  All four warps work in both phases.
-// Receive area of a CTA: [sender slot][128 rows][256 / splits columns + 4], fp32.
-__device__ __forceinline__ void cluster_send_chunks(uint32_t tmem_base, uint8_t* xchg, int g, int lane, int rank,
-                                                    int splits) {
-    const int cpo = (kBN / 32) / splits;                     // chunks per owner
-    const int pitch = cpo * 32 + 4;                          // floats per row of the receive area
-    const uint32_t row_off = (uint32_t)((32 * g + lane) * pitch) * 4u;
-#pragma unroll 1
-    for (int ch = 0; ch < kBN / 32; ++ch) {
-        const int owner = ch / cpo;
-        if (owner == rank) continue;                         // uniform over the warp
-        const int slot = rank < owner ? rank : rank - 1;     // the owner keeps no slot for itself
-        const uint32_t local = ptx::smem_u32(xchg) + (uint32_t)(slot * kBM * pitch) * 4u + row_off +
-                               (uint32_t)((ch - owner * cpo) * 32) * 4u;
-        const uint32_t remote = ptx::map_shared_to_cta(local, (uint32_t)owner);
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
-        ptx::tmem_ld_wait();
-#pragma unroll
-        for (int e = 0; e < 32; e += 4)
-            ptx::st_cluster_v4(remote + (uint32_t)e * 4u, __uint_as_float(r[e]), __uint_as_float(r[e + 1]),
-                               __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-    }
-}
-
 __device__ __forceinline__ void cluster_finish_chunks(uint32_t tmem_base, const uint8_t* xchg, float* stage, int g,
-                                                      int lane, int rank, int splits, int j0, int c0, int Ca, int Cz,
-                                                      float* __restrict__ dw, int accumulate) {
+                                                      int sub, int lane, int rank, int splits, int j0, int c0, int Ca,
+                                                      int Cz, float* __restrict__ dw, int accumulate) {
     const int cpo = (kBN / 32) / splits;
     const int pitch = cpo * 32 + 4;
     const float* mine = reinterpret_cast<const float*>(xchg) + (size_t)(32 * g + lane) * pitch;
     const int rr0 = lane >> 3, q = lane & 7;
 #pragma unroll 1
-    for (int cl = 0; cl < cpo; ++cl) {
+    for (int cl = sub; cl < cpo; cl += kEpiSubs) {
         const int ch = rank * cpo + cl;
         uint32_t r[32];
         ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
@@ -309,7 +297,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, int Ca, int Cz,
              int tiles_n, int splits, int kb_per_split, int kb_total, float* __restrict__ dw, int accumulate,
              float* __restrict__ partial, uint32_t* counters, int32_t* dev_status, int cluster_mode,
-             int grouped_maps) {
+             int grouped_maps, uint32_t wait_limit) {
     extern __shared__ uint8_t smem_raw[];
     // The dynamic window starts at the same offset in every CTA of the kernel, so this rounding gives
     // the same offsets in both CTAs of a cluster (the exchange below maps addresses between them).
@@ -358,7 +346,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
             int issued = 0;
             for (int i = 0; i < nkb && !*abort_flag; ++i) {
                 const int s = i % kStages;
-                if (i >= kStages && !ptx::mbar_wait_spin(&ctl->empty[s], ((i / kStages) - 1) & 1, kWaitLimit)) {
+                if (i >= kStages && !ptx::mbar_wait_spin(&ctl->empty[s], ((i / kStages) - 1) & 1, wait_limit)) {
                     *abort_flag = 1;
                     break;
                 }
@@ -387,12 +375,10 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::make_idesc_bf16(kBM, kBN, true, true);
             constexpr uint32_t kGroupBytes = 64 * kBK * 2;   // one 64-wide M/N group: kBK rows of 128 bytes
-            bool ok = true;
             for (int i = 0; i < nkb; ++i) {
                 const int s = i % kStages;
-                if (*abort_flag || !ptx::mbar_wait_spin(&ctl->full[s], (i / kStages) & 1, kWaitLimit)) {
+                if (*abort_flag || !ptx::mbar_wait_spin(&ctl->full[s], (i / kStages) & 1, wait_limit)) {
                     *abort_flag = 1;
-                    ok = false;
                     break;
                 }
                 ptx::tc_fence_after();
@@ -406,12 +392,12 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
                 }
                 ptx::umma_commit(&ctl->empty[s]);
             }
-            if (ok) ptx::umma_commit(&ctl->accum);
+            ptx::umma_commit(&ctl->accum);   // also after an abort: the barrier then tells when the MMAs in flight are done
         }
     } else {
         // ---------------- epilogue: TMEM -> global ----------------
         ptx::launch_dependents();   // a programmatically launched kernel behind this one may be brought up
-        bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
+        bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, wait_limit);
         ok = __all_sync(kFullMask, ok) && !*abort_flag;
         if (!ok) *abort_flag = 1;
         if (!cluster_mode) {
@@ -421,7 +407,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         uint32_t* done = counters + gridDim.x + tile;
         if (splits > 1) {
             if (threadIdx.x == 64) ctl->finisher = (atomicAdd(tickets, 1u) == (uint32_t)splits - 1) ? 1 : 0;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
         }
         const bool finisher = ctl->finisher != 0;
         if (finisher && splits > 1) {
@@ -434,17 +420,17 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
                 }
                 __threadfence();
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
         }
         if (!*abort_flag) {
             ptx::tc_fence_after();
             float* stage = reinterpret_cast<float*>(smem) + (warp - 2) * kEpiWarpFloats;
-            epilogue_tile_staged(tmem_base, stage, warp & 3, lane, j0, c0, Ca, Cz, split, splits, finisher, dw,
+            epilogue_tile_staged(tmem_base, stage, warp & 3, (warp - 2) >> 2, lane, j0, c0, Ca, Cz, split, splits, finisher, dw,
                                  accumulate, partial);
         }
         if (!finisher) {   // publish the partial plane (also after an abort, so that the finisher's wait ends)
             __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
             if (threadIdx.x == 64) atomicAdd(done, 1u);
         }
         }   // ticket path
@@ -460,17 +446,20 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         const int g = warp & 3;
         if (warp >= 2 && !*abort_flag) {
             ptx::tc_fence_after();
-            cluster_send_chunks(tmem_base, xchg, g, lane, split, splits);
+            cluster_send_chunks(tmem_base, xchg, g, (warp - 2) >> 2, kEpiSubs, lane, split, splits);
         }
         __syncwarp();
         ptx::cluster_sync_all();                                           // every chunk has been delivered
         if (warp >= 2 && !*abort_flag)
-            cluster_finish_chunks(tmem_base, xchg, stage, g, lane, split, splits, j0, c0, Ca, Cz, dw, accumulate);
+            cluster_finish_chunks(tmem_base, xchg, stage, g, (warp - 2) >> 2, lane, split, splits, j0, c0, Ca, Cz, dw, accumulate);
     }
 
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 1) {
+        // after an abort nobody has waited for the MMAs that were already issued: tensor memory is not given
+        // back while they may still write to it (always the full limit here)
+        if (*abort_flag) ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kBN);
     }
@@ -545,12 +534,15 @@ extern "C" dropit_status dropit_weight_grad_workspace(int64_t M, int64_t Ca, int
     if (M < 0 || Ca <= 0 || Cz <= 0 || M * Ca >= ((int64_t)1 << 31)) return DROPIT_ERR_INVALID_ARG;
     if ((dtype != DROPIT_BF16 && dtype != DROPIT_F32) || (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32))
         return DROPIT_ERR_INVALID_ARG;
-    if (workspace_bytes) {   // enough for either variant
-        const size_t a = make_wg_plan(M, Ca, Cz, dtype, format, false).total_bytes;
-        const size_t b = make_wg_plan(M, Ca, Cz, dtype, format, true).total_bytes;
-        *workspace_bytes = a > b ? a : b;
-    }
+    if (workspace_bytes) *workspace_bytes = make_wg_plan(M, Ca, Cz, dtype, format, false).total_bytes;
     return DROPIT_OK;
+}
+
+// DROPIT_WG_PATH=fused makes dropit_weight_grad take the kernel without a scratch wherever it applies
+// (for comparisons; the workspace that dropit_weight_grad_workspace states is then more than is used).
+static bool prefer_fused() {
+    const char* e = std::getenv("DROPIT_WG_PATH");
+    return e && std::strcmp(e, "fused") == 0;
 }
 
 static dropit_status weight_grad_impl(const void* dy, const void* values, const void* meta,
@@ -562,6 +554,7 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     if ((dtype != DROPIT_BF16 && dtype != DROPIT_F32) || (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32))
         return DROPIT_ERR_INVALID_ARG;
     if (!dw || !is_aligned16(dw)) return DROPIT_ERR_INVALID_ARG;
+    if (force_fused && !fused_supported(Ca, Cz, dtype, format)) return DROPIT_ERR_UNSUPPORTED;
     cudaStream_t stream = as_stream(cuda_stream);
     if (M == 0 || k == 0) {   // empty batch or gamma = 1: the gradient is zero
         zero_or_keep_kernel<<<sm_count(), 256, 0, stream>>>(dw, Cz * Ca, accumulate);
@@ -570,21 +563,14 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     if (!dy || !values || !meta || !is_aligned16(dy) || !is_aligned16(values) || !is_aligned16(meta))
         return DROPIT_ERR_INVALID_ARG;
     if (format == DROPIT_FMT_BITMASK && (!offsets || !is_aligned16(offsets))) return DROPIT_ERR_INVALID_ARG;
-    const WgPlan plan = make_wg_plan(M, Ca, Cz, dtype, format, force_fused);
-    if (force_fused && !plan.fused) return DROPIT_ERR_UNSUPPORTED;
+    const WgPlan plan = make_wg_plan(M, Ca, Cz, dtype, format, force_fused || prefer_fused());
+    if (plan.fused)   // one launch, no scratch
+        return launch_wg_tmem(dy, values, meta, offsets, M, Ca, Cz, k, plan.splits, plan.kb_per_split, plan.kb_total, dw,
+                              accumulate, dev_status, stream);
     if (!workspace || !is_aligned16(workspace)) return DROPIT_ERR_INVALID_ARG;
     if (workspace_bytes < plan.total_bytes) return DROPIT_ERR_WORKSPACE;
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
     void* dense = ws + plan.dense_off;
-
-    if (plan.fused) {
-        uint32_t* counters = reinterpret_cast<uint32_t*>(ws + plan.counters_off);
-        float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
-        if (plan.splits > 1 && cudaMemsetAsync(counters, 0, plan.counters_bytes, stream) != cudaSuccess)
-            return DROPIT_ERR_CUDA;
-        return launch_wg_fused(dy, values, meta, offsets, M, Ca, Cz, k, plan.tiles_m, plan.tiles_n, plan.splits,
-                               plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status, stream);
-    }
     dropit_status s = decompress_dispatch(values, meta, offsets, M * Ca, k, dtype, format, dense, stream);
     if (s != DROPIT_OK) return s;
 
@@ -613,12 +599,12 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
     if (plan.splits > 1 && !plan.cluster && cudaMemsetAsync(counters, 0, plan.counters_bytes, stream) != cudaSuccess)
         return DROPIT_ERR_CUDA;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce smem_attr;
+    if (smem_attr.needed()) {
         if (cudaFuncSetAttribute(wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) !=
             cudaSuccess)
             return DROPIT_ERR_CUDA;
-        attr_set = true;
+        smem_attr.mark();
     }
     dim3 grid(plan.tiles_m * plan.tiles_n, plan.splits);
     cudaLaunchConfig_t cfg = {};
@@ -644,7 +630,7 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     }
     if (cudaLaunchKernelEx(&cfg, wg_tc_kernel, map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n, plan.splits,
                            plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status,
-                           plan.cluster ? 1 : 0, grouped ? 1 : 0) != cudaSuccess) {
+                           plan.cluster ? 1 : 0, grouped ? 1 : 0, spin_limit(kWaitLimit)) != cudaSuccess) {
         (void)cudaGetLastError();
         return DROPIT_ERR_CUDA;
     }

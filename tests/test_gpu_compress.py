@@ -177,7 +177,7 @@ def test_repeat_calls_are_bit_identical(cuda_device):
 
 FULL = [di.VITB_FC1, di.VITB_FC2, di.R50_CONV1X1, di.R50_CONV3X3,
         di.with_gamma(di.VITDET_QKV, 0.5), di.with_gamma(di.VITDET_QKV, 0.8), di.VITDET_QKV,
-        di.with_gamma(di.VITDET_FC2, 0.5)]
+        di.with_gamma(di.VITDET_FC2, 0.5), di.with_gamma(di.VITDET_FC2, 0.8), di.VITDET_FC2]
 
 
 @pytest.mark.parametrize("case", FULL, ids=lambda c: c.name)

@@ -27,6 +27,16 @@ SMALL = [
     di.small_linear(8192, 256, 128, "bf16", 0.9),                      # one tile, deep split along tokens
     di.small_linear(200, 2056, 1000, "bf16", 0.9),                     # 72 tiles x 2 splits: cluster of 2, ragged tiles
     di.small_linear(512, 1792, 520, "bf16", 0.9),                      # 35 tiles x 4 splits: cluster of 4, ragged rows
+    # the scratch is produced inside the GEMM kernel (channel counts that are multiples of 64):
+    di.small_linear(131, 192, 64, "bf16", 0.7),                        # ragged last step (n = 24 * 1024 + 576), ragged k-block
+    di.small_linear(333, 320, 192, "bf16", 0.5),                       # two column tiles, the second one partial
+    di.small_linear(700, 256, 256, "bf16", 0.2),                       # dense steps: more values than the look-ahead window
+    di.small_linear(4100, 1024, 1152, "bf16", 0.9),                    # 36 tiles x 4 splits: cluster of 4
+    di.small_linear(2000, 2048, 1152, "bf16", 0.8),                    # 72 tiles x 2 splits: cluster of 2
+    di.small_linear(1500, 1280, 384, "bf16", 0.9),                     # 15 tiles x 9 splits: partial planes + tickets
+    di.small_linear(300, 256, 256, "bf16", 0.5),                       # half of every row retained: runs longer than the value window
+    di.small_linear(777, 384, 200, "bf16", 0.6),                       # ragged tokens and outputs, dense rows
+    di.small_linear(4096, 128, 8, "bf16", 0.95),                       # one channel tile, eight outputs
 ]
 
 
@@ -78,6 +88,10 @@ def test_fused_weight_grad_matches_oracle(cuda_device, case):
     assert torch.allclose(dw, dw2, rtol=1e-4, atol=1e-6 * float(dw2.abs().max()))
     # reproducible run to run
     assert torch.equal(dw, dropit.dropit_weight_grad(dy.to(cuda_device), cache, fused=True))
+    # accumulate adds to what is there
+    out = torch.full_like(dw, 0.25)
+    dropit.dropit_weight_grad(dy.to(cuda_device), cache, out=out, accumulate=True, fused=True)
+    assert torch.allclose(out, dw + 0.25, rtol=1e-6, atol=1e-6)
 
 
 def test_fused_weight_grad_full_size_and_unsupported(cuda_device):
@@ -86,6 +100,11 @@ def test_fused_weight_grad_full_size_and_unsupported(cuda_device):
     dwf = dropit.dropit_weight_grad(di.make_dy(case).to(cuda_device), cache, fused=True)
     dropit.check_device_status(cuda_device)
     assert torch.allclose(dwf, dw, rtol=1e-4, atol=1e-6 * float(dw.abs().max()))
+    rng = np.random.default_rng(1)
+    js, cs = rng.integers(0, case.Cz, 2000), rng.integers(0, case.Ca, 2000)
+    ref = oracle.fc_weight_grad_entries(dyb, bits, keep, case.M, case.Ca, case.Cz, dt, js, cs)
+    err = np.abs(dwf.cpu().numpy()[js, cs] - ref).max() / np.abs(ref).max()
+    assert err <= TIGHT["bf16"], err
     small = di.small_linear(64, 100, 36, "bf16", 0.5)
     c2 = dropit.dropit_compress(di.make_x(small).to(cuda_device), 0.5, "bitmask")
     with pytest.raises(dropit.DropITError):
@@ -106,6 +125,30 @@ def test_accumulate_adds_to_existing_gradient(cuda_device, case):
     assert torch.equal(out2, dw)
 
 
+def test_weight_grad_scratch_needs_no_initialisation(cuda_device):
+    """The workspace (split counters, ready flags of the in-kernel production, dense scratch) may hold
+    anything: bytes of one value, random bytes, or what an earlier call on another tensor left there."""
+    case = di.small_linear(2000, 2048, 1152, "bf16", 0.8)
+    bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
+    dy = di.make_dy(case).to(cuda_device)
+    wb = dropit.dropit_weight_grad_workspace(case.M, case.Ca, case.Cz, dropit.BF16, dropit.FMT_BITMASK, cuda_device)
+    g = torch.Generator(device="cpu").manual_seed(5)
+    fills = [torch.zeros(wb, dtype=torch.uint8), torch.full((wb,), 0xFF, dtype=torch.uint8),
+             torch.randint(0, 256, (wb,), dtype=torch.uint8, generator=g)]
+    for f in fills:
+        ws = f.to(cuda_device)
+        for _ in range(2):     # the second call finds the first call's flags
+            out = dropit.dropit_weight_grad(dy, cache, workspace=ws)
+            dropit.check_device_status(cuda_device)
+            assert torch.equal(out, dw)
+    other = di.small_linear(1000, 2048, 1152, "bf16", 0.5)
+    c2 = dropit.dropit_compress(di.make_x(other).to(cuda_device), other.gamma, "bitmask")
+    ws = torch.empty(wb, dtype=torch.uint8, device=cuda_device)
+    dropit.dropit_weight_grad(di.make_dy(other).to(cuda_device), c2, workspace=ws)
+    assert torch.equal(dropit.dropit_weight_grad(dy, cache, workspace=ws), dw)
+    dropit.check_device_status(cuda_device)
+
+
 def test_weight_grad_is_reproducible(cuda_device):
     case = di.small_linear(8192, 256, 128, "bf16", 0.9)
     bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
@@ -114,7 +157,13 @@ def test_weight_grad_is_reproducible(cuda_device):
         assert torch.equal(dropit.dropit_weight_grad(dy, cache), dw)
 
 
-@pytest.mark.parametrize("case", [di.VITB_FC1, di.VITB_FC2, di.with_gamma(di.VITDET_QKV, 0.8)], ids=lambda c: c.name)
+FULL_SIZE = [di.VITB_FC1, di.VITB_FC2,
+             di.with_gamma(di.VITDET_QKV, 0.5), di.with_gamma(di.VITDET_QKV, 0.8), di.VITDET_QKV,
+             di.with_gamma(di.VITDET_FC1, 0.5), di.VITDET_FC1,
+             di.with_gamma(di.VITDET_FC2, 0.5), di.VITDET_FC2]
+
+
+@pytest.mark.parametrize("case", FULL_SIZE, ids=lambda c: c.name)
 def test_weight_grad_full_size_sampled_entries(cuda_device, case):
     bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
     got = dw.cpu().numpy()

@@ -61,6 +61,37 @@ def test_static_scratch_variant_matches_the_regular_entry_point_twice_in_a_row(c
     dropit.check_device_status(cuda_device)
 
 
+def test_static_scratch_variant_allocates_no_device_memory(cuda_device):
+    """With every buffer in place beforehand, the call itself must leave the device's memory as it was: nothing
+    taken from the driver (free bytes as the driver reports them) and nothing from torch's allocator."""
+    lib = _lib.load()
+    case = di.small_linear(3000, 768, 1, "bf16", 0.9)
+    x = di.make_x(case).to(cuda_device)
+    n = x.numel()
+    vb, mb, ob, _ = dropit.dropit_cache_sizes(n, 0.9, dropit.BF16, dropit.FMT_BITMASK)
+    values = torch.empty(vb // 2, dtype=torch.bfloat16, device=cuda_device)
+    meta = torch.empty(mb // 4, dtype=torch.int32, device=cuda_device)
+    offsets = torch.empty(ob // 4, dtype=torch.int32, device=cuda_device)
+    status = torch.zeros(4, dtype=torch.int32, device=cuda_device)
+    stream = ctypes.c_void_p(torch.cuda.current_stream(cuda_device).cuda_stream)
+
+    def call():
+        return lib.dropit_compress_static(_ptr(x), n, 0.9, dropit.FMT_BITMASK, _ptr(values), _ptr(meta), _ptr(offsets),
+                                          _ptr(status), stream)
+
+    assert call() == 0          # the first call on a device looks up the scratch address and sets kernel attributes
+    torch.cuda.synchronize(cuda_device)
+    free0, _ = torch.cuda.mem_get_info(cuda_device)
+    alloc0, reserved0 = torch.cuda.memory_allocated(cuda_device), torch.cuda.memory_reserved(cuda_device)
+    for _ in range(3):
+        assert call() == 0
+    torch.cuda.synchronize(cuda_device)
+    free1, _ = torch.cuda.mem_get_info(cuda_device)
+    assert free0 - free1 < (1 << 20)      # (device-wide figure: allow for noise below one allocation granule)
+    assert torch.cuda.memory_allocated(cuda_device) == alloc0 and torch.cuda.memory_reserved(cuda_device) == reserved0
+    assert int(status[0].item()) == 0
+
+
 def test_static_scratch_variant_rejects_oversize_and_bad_arguments(cuda_device):
     lib = _lib.load()
     null = ctypes.c_void_p(0)
