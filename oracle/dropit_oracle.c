@@ -18,7 +18,12 @@
  *                          Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC'11) and
  *                          the k highest ranks are retained, ties to the lower flat index
  *
- * Floating point: products and sums in double, one rounding to float at the end.
+ *   - producer in front    Sec. 3.5 (the layers whose outputs are the conv / fc inputs: activations and
+ *     of the path          normalisations keep their own caches): the element-wise producer y = act(x) of a bf16
+ *                          tensor stated as a table over all 65536 bit patterns (act evaluated in double,
+ *                          rounded once to bf16, ties to even), and the histogram of the ordering keys of y
+ *
+ * Floating point: products and sums in double; results are returned as double.
  * Elements are passed as raw bits (uint16 for bf16, uint32 for fp32); the
  * ordering key of an element is its bits with the sign bit cleared, so
  * -0 == +0, Inf is above every finite value and NaN patterns are above Inf.
@@ -28,7 +33,9 @@
  * sort; closed-form keep counts; closed-form Gaussian quantiles; all-equal and
  * strictly-monotone tensors; numpy float64 matmul at gamma = 0; torch's
  * float64 conv weight gradient; 1x1 conv == FC on the transposed view; the
- * Philox test vectors printed with the generator's reference distribution.
+ * Philox test vectors printed with the generator's reference distribution; the
+ * bf16 rounding against exact rational arithmetic, the GELU table against an
+ * independent erf and the same exact rounding, the ReLU table in closed form.
  */
 #include <math.h>
 #include <stdint.h>
@@ -342,6 +349,72 @@ void oracle_conv_weight_grad_entries(const void* dy, const void* x, const uint8_
                 }
         out[s] = acc;
     }
+}
+
+/* ---- the producer in front of the path (Sec. 3.5) ------------------------ */
+
+/* A double rounded once to bf16 (8 significant bits, the exponent range of fp32), ties to even.
+ * |v| = m * 2^(e-7) with 128 <= m < 256 is scaled so that rint() (ties to even in the default
+ * rounding mode; the scaling by a power of two is exact) does the rounding.  Subnormal results
+ * use the fixed scale 2^-133.  NaN gives the one pattern 0x7FC0. */
+uint16_t oracle_round_to_bf16(double v) {
+    if (v != v) return 0x7FC0;
+    const uint16_t sign = signbit(v) ? 0x8000 : 0;
+    const double a = fabs(v);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return (uint16_t)(sign | 0x7F80);
+    int e2;
+    (void)frexp(a, &e2);              /* a = f * 2^e2, 0.5 <= f < 1  ->  floor(log2 a) = e2 - 1 */
+    int e = e2 - 1;
+    if (e < -126) {                   /* subnormal range of bf16: units of 2^-133 */
+        const double r = rint(ldexp(a, 133));      /* 0 .. 128 */
+        return (uint16_t)(sign | (uint16_t)r);     /* 128 = the smallest normal: exponent field 1, mantissa 0 */
+    }
+    double r = rint(ldexp(a, 7 - e)); /* 128 .. 256 */
+    if (r == 256.0) {
+        r = 128.0;
+        e += 1;
+    }
+    const int E = e + 127;
+    if (E >= 255) return (uint16_t)(sign | 0x7F80);
+    return (uint16_t)(sign | (uint16_t)(E << 7) | ((uint16_t)r - 128));
+}
+
+#define ACT_IDENTITY 0
+#define ACT_RELU 1
+#define ACT_GELU 2
+
+/* y = act(x) for every bf16 bit pattern b (table[b] = bits of y).
+ *   identity: the bits themselves.
+ *   ReLU: max(x, 0): x for x > 0, +0 for x <= 0 (also for -0); NaN patterns pass through unchanged.
+ *   GELU: x * Phi(x) with Phi(x) = erfc(-x / sqrt 2) / 2 in double (the form that keeps its digits for
+ *         negative x, where 1 + erf(x / sqrt 2) cancels), rounded once; NaN patterns pass through unchanged,
+ *         and -Inf (whose product Inf * 0 is not a number) gives 0x7FC0. */
+void oracle_activation_table(int act, uint16_t* table) {
+    for (uint32_t b = 0; b < 65536; ++b) {
+        const uint16_t key = (uint16_t)(b & 0x7FFF);
+        uint16_t y;
+        if (act == ACT_IDENTITY || key > 0x7F80) {
+            y = (uint16_t)b;
+        } else if (act == ACT_RELU) {
+            y = ((b & 0x8000) || key == 0) ? 0 : (uint16_t)b;
+        } else {
+            const double x = bf16_bits_to_double((uint16_t)b);
+            y = oracle_round_to_bf16(x * (0.5 * erfc(-x / sqrt(2.0))));
+        }
+        table[b] = y;
+    }
+}
+
+/* y[i] = table[x[i]] */
+void oracle_apply_table(const uint16_t* table, const uint16_t* x, int64_t n, uint16_t* y) {
+    for (int64_t i = 0; i < n; ++i) y[i] = table[x[i]];
+}
+
+/* Histogram of the ordering keys of a bf16 tensor: hist[key] = #{i : bits_i with the sign cleared = key}. */
+void oracle_key_histogram_bf16(const uint16_t* x, int64_t n, uint64_t* hist /* 32768 */) {
+    memset(hist, 0, 32768 * sizeof(uint64_t));
+    for (int64_t i = 0; i < n; ++i) hist[x[i] & 0x7FFF] += 1;
 }
 
 int oracle_num_threads(void) {

@@ -18,10 +18,12 @@ __all__ = [
     "encode_bitmask", "encode_index32", "pack_values", "chunk_offsets", "recover_from_bitmask",
     "recover_from_index32", "fc_weight_grad", "fc_weight_grad_entries", "conv_weight_grad",
     "conv_weight_grad_entries", "num_threads", "bits_to_float64", "philox4x32_10", "random_ranks", "random_k",
+    "ACT_IDENTITY", "ACT_RELU", "ACT_GELU", "round_to_bf16", "activation_table", "apply_table", "key_histogram_bf16",
 ]
 
 BF16 = 0
 F32 = 1
+ACT_IDENTITY, ACT_RELU, ACT_GELU = 0, 1, 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "dropit_oracle.c")
@@ -53,6 +55,8 @@ def _load():
             lib.oracle_min_k.restype = ctypes.c_int
             lib.oracle_random_k.restype = ctypes.c_int
             lib.oracle_num_threads.restype = ctypes.c_int
+            lib.oracle_round_to_bf16.restype = ctypes.c_uint16
+            lib.oracle_round_to_bf16.argtypes = [ctypes.c_double]
             _lib = lib
     return _lib
 
@@ -272,3 +276,34 @@ def conv_weight_grad_entries(dy_bits, x_bits, keep, B, Ca, H, W, Cz, R, S, strid
                                             _i64(Cz), _i64(R), _i64(S), _i64(stride), _i64(pad), ctypes.c_int(dtype),
                                             _p(js), _p(cs), _p(us), _p(vs), _i64(js.size), _p(out))
     return out
+
+
+def round_to_bf16(v: float) -> int:
+    """A double rounded once to bf16, ties to even; the result's bits."""
+    return int(_load().oracle_round_to_bf16(float(v)))
+
+
+def activation_table(act: int) -> np.ndarray:
+    """The element-wise producer in front of a conv / fc input (Sec. 3.5) as a table over all bf16 bit
+    patterns: table[b] = bits of act(value of b), act in double, rounded once."""
+    table = np.empty(65536, np.uint16)
+    _load().oracle_activation_table(ctypes.c_int(int(act)), _p(table))
+    return table
+
+
+def apply_table(table: np.ndarray, x_bits: np.ndarray) -> np.ndarray:
+    """y[i] = table[x[i]] on raw bf16 bits."""
+    table = _check_bits(table, BF16)
+    x = _check_bits(x_bits, BF16)
+    assert table.size == 65536
+    y = np.empty_like(x)
+    _load().oracle_apply_table(_p(table), _p(x), _i64(x.size), _p(y))
+    return y
+
+
+def key_histogram_bf16(x_bits: np.ndarray) -> np.ndarray:
+    """hist[key] = number of elements whose bits with the sign cleared equal key (32768 bins)."""
+    x = _check_bits(x_bits, BF16)
+    hist = np.zeros(32768, np.uint64)
+    _load().oracle_key_histogram_bf16(_p(x), _i64(x.size), _p(hist))
+    return hist
