@@ -60,6 +60,10 @@ typedef enum {
 
 typedef enum { DROPIT_BF16 = 0, DROPIT_F32 = 1 } dropit_dtype;
 typedef enum { DROPIT_FMT_BITMASK = 0, DROPIT_FMT_INDEX32 = 1 } dropit_format;
+/* Element-wise producers of a layer input (see dropit_produce): y = x, y = max(x, 0), or y = table[x]. */
+typedef enum { DROPIT_ACT_IDENTITY = 0, DROPIT_ACT_RELU = 1, DROPIT_ACT_TABLE = 2 } dropit_activation;
+/* Tables that dropit_activation_table can build. */
+typedef enum { DROPIT_TABLE_IDENTITY = 0, DROPIT_TABLE_RELU = 1, DROPIT_TABLE_GELU = 2 } dropit_table_kind;
 
 /* Elements covered by one entry of the offsets table. */
 #define DROPIT_CHUNK 128
@@ -132,6 +136,40 @@ dropit_status dropit_compress_random_workspace(int64_t n, double gamma, size_t* 
 dropit_status dropit_compress_random(const void* x, int64_t n, double gamma, uint64_t seed, dropit_dtype dtype,
                                      dropit_format format, void* values, void* meta, uint32_t* offsets,
                                      void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * The producer in front of the path.  Sec. 3.5: the inputs of conv / fc layers are the outputs of
+ * activation and normalisation layers, which keep their own caches; the tensor that such a layer
+ * writes is the tensor that DropIT compresses next.  dropit_produce is that element-wise layer for
+ * bf16 tensors, fused with the first half of the selection: it reads x once, writes y = act(x),
+ * and on the way takes the selection statistics of y (the threshold band from a sample, the band
+ * histograms and the counts above the band, per warp and per CTA of the selection kernel's work
+ * partition) into `prep`.  dropit_compress_prepared then produces exactly the cache that
+ * dropit_compress(y, ...) would, with ONE read of y: no sample step, no first pass, no grid barrier.
+ *
+ *   dropit_activation_table: table[b] (device, 65536 uint16) = bits of f(value of bf16 pattern b),
+ *     f evaluated in double and rounded once to bf16 (ties to even).  kinds: identity, ReLU
+ *     (max(x, 0); -0 -> +0; NaN patterns pass), GELU (x Phi(x), Phi(x) = erfc(-x / sqrt 2) / 2; NaN
+ *     patterns pass; -Inf gives the NaN pattern 0x7FC0).  Any other element-wise function can be
+ *     supplied as a table built by the caller.
+ *   dropit_produce: x [device, n bf16, read only]; act: DROPIT_ACT_IDENTITY (y may be NULL: statistics
+ *     only), DROPIT_ACT_RELU, or DROPIT_ACT_TABLE with `table` [device]; y [device, n bf16, written]
+ *     must not be x (every CTA samples x while others already write y); prep [device, >=
+ *     dropit_produce_workspace bytes, written, need not be initialised]; gamma: the drop ratio the
+ *     statistics are taken for.  No device-side waits.
+ *   dropit_compress_prepared: same arguments, outputs and selection rule as dropit_compress with dtype
+ *     DROPIT_BF16, plus `prep` as written by dropit_produce for the same tensor, n and gamma.  If the
+ *     statistics do not fit this call (other n / gamma / device, a tensor too small to be sampled, a
+ *     threshold outside the sampled band) the call silently does the whole selection itself, so the
+ *     result never depends on `prep`; `workspace` as for dropit_compress.
+ */
+dropit_status dropit_activation_table(dropit_table_kind kind, uint16_t* table, void* cuda_stream);
+dropit_status dropit_produce_workspace(int64_t n, size_t* prep_bytes);
+dropit_status dropit_produce(const void* x, int64_t n, double gamma, dropit_activation act, const uint16_t* table,
+                             void* y, void* prep, size_t prep_bytes, void* cuda_stream);
+dropit_status dropit_compress_prepared(const void* y, int64_t n, double gamma, dropit_format format, void* values,
+                                       void* meta, uint32_t* offsets, const void* prep, size_t prep_bytes,
+                                       void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
 /* Largest tensor (elements) that dropit_compress_static accepts. */
 #define DROPIT_STATIC_MAX_ELEMS (1 << 28)

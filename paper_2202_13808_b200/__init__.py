@@ -10,5 +10,6 @@ from .api import (  # noqa: F401
     dropit_cache_sizes, dropit_compress, dropit_compress_random, dropit_compress_random_workspace, dropit_conv_weight_grad, dropit_conv_weight_grad_workspace,
     dropit_decompress, dropit_keep_count, dropit_launch_count, dropit_status_string, dropit_version, dropit_weight_grad,
     dropit_weight_grad_workspace, check_device_status, library_path,
+    dropit_activation_table, dropit_produce, dropit_produce_workspace, dropit_compress_prepared,
 )
 from .nn import DropITConv2d, DropITConv2dFn, DropITLinear, DropITLinearFn, convert_linear_layers  # noqa: F401

@@ -25,6 +25,10 @@ SIGNATURES = {
     "dropit_compress_random_workspace": (c_int, [c_i64, c_dbl, p_sz]),
     "dropit_compress_random": (c_int, [c_vp, c_i64, c_dbl, ctypes.c_uint64, c_int, c_int, c_vp, c_vp, c_vp, c_vp, c_sz,
                                        c_vp, c_vp]),
+    "dropit_activation_table": (c_int, [c_int, c_vp, c_vp]),
+    "dropit_produce_workspace": (c_int, [c_i64, p_sz]),
+    "dropit_produce": (c_int, [c_vp, c_i64, c_dbl, c_int, c_vp, c_vp, c_vp, c_sz, c_vp]),
+    "dropit_compress_prepared": (c_int, [c_vp, c_i64, c_dbl, c_int, c_vp, c_vp, c_vp, c_vp, c_sz, c_vp, c_sz, c_vp, c_vp]),
     "dropit_compress_static_scratch_bytes": (c_sz, []),
     "dropit_compress_static": (c_int, [c_vp, c_i64, c_dbl, c_int, c_vp, c_vp, c_vp, c_vp, c_vp]),
     "dropit_decompress": (c_int, [c_vp, c_vp, c_vp, c_i64, c_i64, c_int, c_int, c_vp, c_vp]),

@@ -150,6 +150,86 @@ def dropit_compress(x: torch.Tensor, gamma: float, fmt="bitmask", workspace: Opt
     return DropITCache(values, meta, offsets, n, k, tuple(x.shape), x.dtype, fmt, float(gamma))
 
 
+ACT_IDENTITY, ACT_RELU, ACT_TABLE = 0, 1, 2
+TABLE_IDENTITY, TABLE_RELU, TABLE_GELU = 0, 1, 2
+_TABLE_KIND = {"identity": TABLE_IDENTITY, "relu": TABLE_RELU, "gelu": TABLE_GELU}
+_tables = {}
+
+
+def dropit_activation_table(kind: str, device) -> torch.Tensor:
+    """bf16 -> bf16 table of an element-wise activation over all 65536 bit patterns (int16 tensor on `device`),
+    every entry evaluated in double and rounded once; built on the device the first time it is asked for."""
+    device = torch.device(device)
+    key = (kind, device.type, _device_index(device))
+    if key not in _tables:
+        t = torch.empty(65536, dtype=torch.int16, device=device)
+        with _on_device(device):
+            code = _lib.load().dropit_activation_table(_TABLE_KIND[kind], _ptr(t), _stream_ptr(device))
+        _check(code, "dropit_activation_table")
+        _tables[key] = t
+    return _tables[key]
+
+
+@functools.lru_cache(maxsize=4096)
+def dropit_produce_workspace(n: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(_lib.load().dropit_produce_workspace(int(n), ctypes.byref(out)), "dropit_produce_workspace")
+    return int(out.value)
+
+
+def dropit_produce(x: torch.Tensor, gamma: float, act: str = "identity", table: Optional[torch.Tensor] = None,
+                   want_y: bool = True):
+    """The element-wise layer in front of a conv / fc input (Sec. 3.5) fused with the first half of the selection:
+    returns (y, prep) with y = act(x) (None when act is "identity" and want_y is False) and prep the selection
+    statistics of y for drop ratio gamma, to be handed to dropit_compress_prepared.
+    act: "identity", "relu", "gelu", or "table" with an int16 tensor of 65536 bf16 patterns."""
+    _require_cuda(x, "x")
+    if x.dtype != torch.bfloat16:
+        raise TypeError("dropit_produce takes bf16 tensors")
+    dev = x.device
+    if act == "gelu":
+        table, code_act = dropit_activation_table("gelu", dev), ACT_TABLE
+    elif act == "table":
+        if table is None or table.numel() != 65536 or table.dtype != torch.int16 or table.device != dev:
+            raise ValueError("table must be an int16 tensor of 65536 bf16 patterns on the input's device")
+        code_act = ACT_TABLE
+    else:
+        code_act = {"identity": ACT_IDENTITY, "relu": ACT_RELU}[act]
+    n = x.numel()
+    y = torch.empty_like(x) if (want_y or code_act != ACT_IDENTITY) else None
+    prep = torch.empty(max(dropit_produce_workspace(n), 16), dtype=torch.uint8, device=dev)
+    with _on_device(dev):
+        code = _lib.load().dropit_produce(_ptr(x), n, float(gamma), code_act, _ptr(table), _ptr(y), _ptr(prep),
+                                          prep.numel(), _stream_ptr(dev))
+    _check(code, "dropit_produce")
+    return y, prep
+
+
+def dropit_compress_prepared(y: torch.Tensor, gamma: float, prep: torch.Tensor, fmt="bitmask",
+                             workspace: Optional[torch.Tensor] = None) -> DropITCache:
+    """dropit_compress of a tensor whose selection statistics dropit_produce has already taken: one read of y."""
+    _require_cuda(y, "y")
+    if y.dtype != torch.bfloat16:
+        raise TypeError("dropit_compress_prepared takes bf16 tensors")
+    lib = _lib.load()
+    fmt = _FMT_CODE[fmt]
+    n = y.numel()
+    vb, mb, ob, wb = dropit_cache_sizes(n, gamma, BF16, fmt)
+    k = dropit_keep_count(n, gamma)
+    dev = y.device
+    values = torch.empty(vb // 2, dtype=torch.bfloat16, device=dev)
+    meta = torch.empty(mb // 4, dtype=torch.int32, device=dev)
+    offsets = torch.empty(ob // 4, dtype=torch.int32, device=dev)
+    if workspace is None or workspace.numel() < wb:
+        workspace = torch.empty(max(wb, 16), dtype=torch.uint8, device=dev)
+    with _on_device(dev):
+        code = lib.dropit_compress_prepared(_ptr(y), n, float(gamma), fmt, _ptr(values), _ptr(meta), _ptr(offsets),
+                                            _ptr(prep), prep.numel(), _ptr(workspace), workspace.numel(),
+                                            _ptr(_status_word(dev)), _stream_ptr(dev))
+    _check(code, "dropit_compress_prepared")
+    return DropITCache(values, meta, offsets, n, k, tuple(y.shape), y.dtype, fmt, float(gamma))
+
+
 @functools.lru_cache(maxsize=4096)
 def dropit_compress_random_workspace(n: int, gamma: float) -> int:
     out = ctypes.c_size_t(0)

@@ -91,6 +91,33 @@ static FusedPlan make_fused_plan(int64_t n) {
 
 size_t fused_compress_workspace_bytes(int64_t n) { return make_fused_plan(n).total_bytes; }
 
+// ---------------------------------------------------------------------------------------------
+// Statistics handed from the producer of a tensor to its compression (produce_kernel below writes them while
+// it writes the tensor, fused_compress_kernel then skips its sample step, its first read and its grid barrier):
+//   header | per-CTA rows [grid][kRowWords] | per-warp band histograms [grid][32 warps][kPrepWarpWords]
+// A row and a per-warp record hold what phase 1 of the selection kernel would have left in shared memory.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kPrepMagic = 0xD20917F1u;
+constexpr int kPrepWarpWords = kWarpBins + 2;                  // band bins, #{key > hi}, pad
+struct PrepHeader {
+    uint32_t magic, valid;               // valid: the tensor was sampled and the band fits the per-warp histograms
+    uint32_t lo, hi;                     // the band of keys around the threshold
+    uint32_t grid, blocks_per_warp;      // the work partition the statistics were taken under
+    unsigned long long n, k;
+    uint32_t reserved[6];
+};
+static_assert(sizeof(PrepHeader) == 64, "PrepHeader layout");
+__host__ __device__ inline const uint32_t* prep_rows(const unsigned char* prep) {
+    return reinterpret_cast<const uint32_t*>(prep + sizeof(PrepHeader));
+}
+__host__ __device__ inline const uint32_t* prep_warp_hist(const unsigned char* prep, uint32_t grid) {
+    return prep_rows(prep) + (size_t)grid * kRowWords;
+}
+static size_t prep_bytes_for(int64_t n) {
+    const FusedPlan p = make_fused_plan(n);
+    return sizeof(PrepHeader) + (size_t)p.grid * kRowWords * 4 + (size_t)p.grid * kFusedWarps * kPrepWarpWords * 4;
+}
+
 __device__ __forceinline__ uint32_t ptx_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
@@ -156,7 +183,7 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
 // %globaltimer at each stamp.  Off in normal builds.
 #ifdef DROPIT_PHASE_TIMING
 __device__ __forceinline__ void phase_stamp(FusedState* st, int i) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (st != nullptr && blockIdx.x == 0 && threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
         reinterpret_cast<unsigned long long*>(st->reserved)[i] = t;
@@ -172,9 +199,12 @@ __device__ __forceinline__ void phase_stamp(FusedState*, int) {}
 // same band without any exchange.  `bins`: kKeySpace counters in shared memory; band[0..1] = lo, hi.
 // Ends with a block-wide barrier.
 // ---------------------------------------------------------------------------------------------
-template <typename AfterLoads>
+// `map`: applied to every sampled vector before its keys are taken (the identity for the selection kernel;
+// the producer kernel brackets the threshold of act(x), so it maps the sample through act).
+template <typename AfterLoads, typename Map>
 __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t n, unsigned long long k, uint32_t* bins,
-                                            uint32_t* s_warp, uint32_t* band, FusedState* st, AfterLoads after_loads) {
+                                            uint32_t* s_warp, uint32_t* band, FusedState* st, AfterLoads after_loads,
+                                            Map map) {
     // after_loads: called once by every thread, after the sample has been counted (or at once when there is no sample)
     const int64_t nvec = n / 8;
     const bool sampled = n >= kSampleMinElems;
@@ -202,7 +232,7 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
 #pragma unroll
         for (int r = 0; r < kSampleVecs / kFusedThreads; ++r) {
             uint32_t key[8];
-            keys_of(sv[r], key);
+            keys_of(map(sv[r]), key);
 #pragma unroll
             for (int e = 0; e < 8; ++e) atomicAdd(&bins[key[e] >> 1], 1u << ((key[e] & 1u) * 16));
         }
@@ -432,7 +462,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long k, int blocks_per_warp, uint32_t epoch,
                       unsigned char* ws, size_t hist_off0, size_t hist_off1, size_t agg_off, size_t rows_off,
                       uint16_t* __restrict__ values, uint32_t* __restrict__ mask, int32_t* __restrict__ indices,
-                      uint32_t* __restrict__ offsets, int32_t* dev_status, int spin_max) {
+                      uint32_t* __restrict__ offsets, int32_t* dev_status, int spin_max, const unsigned char* prep) {
     // shared memory: [input ring, 128 KB | general path: full key histogram]
     //                [phase 3: per-warp value staging, 64 KB | sample step: 16-bit key histogram]
     //                [control block of phases 1-2]
@@ -475,8 +505,25 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     }
     barrier_open(&st->barrier, epoch);
     // the first super-block of the run is requested while the sample is evaluated, which hides its latency
-    bool prefetched = true;
-    sample_band(x, n, k, sample_bins, sh.warp, sh.band, st, [&] { issue_sb(sb0, 0); });
+    const PrepHeader* ph = reinterpret_cast<const PrepHeader*>(prep);
+    // statistics handed over by the producer kernel are used when they describe exactly this call
+    const bool prepared = prep != nullptr && ph->magic == kPrepMagic && ph->valid != 0 && ph->n == (unsigned long long)n &&
+                          ph->k == k && ph->grid == gridDim.x && ph->blocks_per_warp == (uint32_t)blocks_per_warp;
+    if (prepared) {
+        if (threadIdx.x == 0) {
+            sh.band[0] = ph->lo;
+            sh.band[1] = ph->hi;
+        }
+        const uint32_t* wh = prep_warp_hist(prep, ph->grid) + (size_t)blockIdx.x * kFusedWarps * kPrepWarpWords;
+        for (int i = threadIdx.x; i < kFusedWarps * kWarpBins; i += blockDim.x)
+            (&sh.whist[0][0])[i] = wh[(i / kWarpBins) * kPrepWarpWords + (i % kWarpBins)];
+        if (threadIdx.x < kFusedWarps) sh.w_hi[threadIdx.x] = wh[threadIdx.x * kPrepWarpWords + kWarpBins];
+        rows = const_cast<uint32_t*>(prep_rows(prep));
+        __syncthreads();
+    } else {
+        sample_band(x, n, k, sample_bins, sh.warp, sh.band, st, [&] { issue_sb(sb0, 0); }, [](const uint4& v) { return v; });
+    }
+    bool prefetched = !prepared;
     uint32_t lo = sh.band[0], hi = sh.band[1];
     uint32_t T = 0, q = 0;
     uint32_t run_gt = 0, run_eq = 0;   // this warp's exclusive prefix (absolute)
@@ -490,153 +537,157 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         const uint32_t width = hi - lo;
         const bool narrow = width < (uint32_t)kWarpBins;   // uniform over the grid
         uint32_t* ghist = reinterpret_cast<uint32_t*>(ws + (attempt == 0 ? hist_off0 : hist_off1));
-        // ---------------- phase 1: band histogram ----------------
-        if (narrow) {
-            for (int i = threadIdx.x; i < kFusedWarps * kWarpBins; i += blockDim.x) (&sh.whist[0][0])[i] = 0;
-        } else {
-            if (prefetched) {   // the histogram takes the ring's memory: let the requested blocks land first
-                asm volatile("cp.async.wait_all;" ::: "memory");
-                __syncthreads();
-            }
-            for (uint32_t i = threadIdx.x; i <= width; i += blockDim.x) bins[i] = 0;
-        }
-        __syncthreads();
-        uint32_t* hist = narrow ? sh.whist[warp] : bins;
-        const uint32_t c_hi = ge_const(hi + 1), c_lo = ge_const(lo);
-        uint32_t cnt_hi = 0, cnt_lo = 0;   // keys above the band / keys equal to lo
-        auto count_vec = [&](const uint4& v, int nvalid) {
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-            uint32_t a[4], inb[4], any = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t m = w[i] & 0x7FFF7FFFu;
-                a[i] = m + c_hi;                       // bit 15 of a half: key > hi
-                inb[i] = (m + c_lo) & ~a[i];           // bit 15 of a half: lo <= key <= hi
-                any |= inb[i];
-            }
-            // keys above the band: one popc per pair of words (the flag bytes gathered by prmt)
-            cnt_hi += __popc(__byte_perm(a[0], a[1], 0x7531) & 0x80808080u) +
-                      __popc(__byte_perm(a[2], a[3], 0x7531) & 0x80808080u);
-            if (any & kHiBits) {   // a few percent of the elements: the band histogram
-                // one pass per in-band element of the lane's vector (a warp needs about two passes), instead
-                // of a divergent test per word and half
-                uint32_t pending = (flags4(inb[0], inb[1]) | (flags4(inb[2], inb[3]) << 4)) & ((1u << nvalid) - 1u);
-                while (pending) {
-                    const uint32_t e = (uint32_t)__ffs(pending) - 1u;
-                    pending &= pending - 1u;
-                    const uint32_t wlo = (e & 2u) ? w[1] : w[0], whi = (e & 2u) ? w[3] : w[2];
-                    const uint32_t ws = (e & 4u) ? whi : wlo;
-                    const uint32_t key = ((e & 1u) ? (ws >> 16) : ws) & 0x7FFFu;
-                    const uint32_t d = key - lo;
-                    if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
+        // With the producer's statistics the band histograms, the per-warp counts and the per-CTA rows of the
+        // first attempt are already there: no first read of the tensor, no grid barrier.
+        if (!(prepared && attempt == 0)) {
+            // ---------------- phase 1: band histogram ----------------
+            if (narrow) {
+                for (int i = threadIdx.x; i < kFusedWarps * kWarpBins; i += blockDim.x) (&sh.whist[0][0])[i] = 0;
+            } else {
+                if (prefetched) {   // the histogram takes the ring's memory: let the requested blocks land first
+                    asm volatile("cp.async.wait_all;" ::: "memory");
+                    __syncthreads();
                 }
+                for (uint32_t i = threadIdx.x; i <= width; i += blockDim.x) bins[i] = 0;
             }
-        };
-        if (narrow) {
-            // stream the run through the ring, one super-block ahead
-            if (!prefetched) issue_sb(sb0, 0);
-            int slot = 0;
-            auto count_sb = [&](int64_t sb, auto full_tag) {
-                constexpr bool FULL = decltype(full_tag)::value;
-                issue_sb(sb + 1, slot ^ 1);
-                sb_wait();
-                __syncwarp();   // the lane reads vectors that other lanes copied
-                const uint32_t own = ring_own + slot * kSbBytes;
-                uint32_t w[16];
-                sb_read(own, rot, w);
-                uint32_t hi_flags = 0, pending = 0;
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {   // four words = eight elements at a time
-                    uint32_t a[4], b[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t m = w[4 * g + i] & 0x7FFF7FFFu;
-                        a[i] = m + c_hi;                   // bit 15 of a half: key > hi
-                        b[i] = (m + c_lo) & ~a[i];         // bit 15 of a half: lo <= key <= hi
+            __syncthreads();
+            uint32_t* hist = narrow ? sh.whist[warp] : bins;
+            const uint32_t c_hi = ge_const(hi + 1), c_lo = ge_const(lo);
+            uint32_t cnt_hi = 0, cnt_lo = 0;   // keys above the band / keys equal to lo
+            auto count_vec = [&](const uint4& v, int nvalid) {
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                uint32_t a[4], inb[4], any = 0;
+    #pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t m = w[i] & 0x7FFF7FFFu;
+                    a[i] = m + c_hi;                       // bit 15 of a half: key > hi
+                    inb[i] = (m + c_lo) & ~a[i];           // bit 15 of a half: lo <= key <= hi
+                    any |= inb[i];
+                }
+                // keys above the band: one popc per pair of words (the flag bytes gathered by prmt)
+                cnt_hi += __popc(__byte_perm(a[0], a[1], 0x7531) & 0x80808080u) +
+                          __popc(__byte_perm(a[2], a[3], 0x7531) & 0x80808080u);
+                if (any & kHiBits) {   // a few percent of the elements: the band histogram
+                    // one pass per in-band element of the lane's vector (a warp needs about two passes), instead
+                    // of a divergent test per word and half
+                    uint32_t pending = (flags4(inb[0], inb[1]) | (flags4(inb[2], inb[3]) << 4)) & ((1u << nvalid) - 1u);
+                    while (pending) {
+                        const uint32_t e = (uint32_t)__ffs(pending) - 1u;
+                        pending &= pending - 1u;
+                        const uint32_t wlo = (e & 2u) ? w[1] : w[0], whi = (e & 2u) ? w[3] : w[2];
+                        const uint32_t ws = (e & 4u) ? whi : wlo;
+                        const uint32_t key = ((e & 1u) ? (ws >> 16) : ws) & 0x7FFFu;
+                        const uint32_t d = key - lo;
+                        if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
                     }
-                    // above the band only the count matters: the flag bytes of all 16 words share one word
-                    hi_flags |= ((__byte_perm(a[0], a[1], 0x7531) & 0x80808080u) >> (2 * g)) |
-                                ((__byte_perm(a[2], a[3], 0x7531) & 0x80808080u) >> (2 * g + 1));
-                    pending |= flags8(b[0], b[1], b[2], b[3]) << ((g ^ rot) << 3);
                 }
-                cnt_hi += __popc(hi_flags);
-                if constexpr (!FULL) pending &= valid_mask32(sb * kSbElems + lane * 32, n);   // zero padding is no data
-                while (pending) {   // a few percent of the elements: the band histogram (their order is irrelevant)
-                    const uint32_t e = top_bit(pending);
-                    pending ^= 1u << e;
-                    const uint32_t d = (lds_u16(own + 2u * e) & 0x7FFFu) - lo;
-                    if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
-                }
-                __syncwarp();   // every lane is done with the slot before it is refilled
-                slot ^= 1;
             };
-            int64_t sb = sb0;
-            for (; sb < sb_full_end; ++sb) count_sb(sb, std::true_type{});
-            for (; sb < sb1; ++sb) count_sb(sb, std::false_type{});
-            asm volatile("cp.async.wait_all;" ::: "memory");
-        } else {
-            int64_t blk = blk0;
-            for (; blk + kP1Blocks <= blk1; blk += kP1Blocks) {   // 4 loads per lane in flight
-                uint4 va[kP1Blocks][kVpl];
-                int na[kP1Blocks][kVpl];
-#pragma unroll
-                for (int u = 0; u < kP1Blocks; ++u) load_block(x, blk + u, lane, nvec_full, n, va[u], na[u]);
-#pragma unroll
-                for (int u = 0; u < kP1Blocks; ++u)
-#pragma unroll
-                    for (int j = 0; j < kVpl; ++j) count_vec(va[u][j], na[u][j]);
-            }
-            for (; blk < blk1; ++blk) {
-                uint4 va[kVpl];
-                int na[kVpl];
-                load_block(x, blk, lane, nvec_full, n, va, na);
-#pragma unroll
-                for (int j = 0; j < kVpl; ++j) count_vec(va[j], na[j]);
-            }
-        }
-        prefetched = false;
-        phase_stamp(st, 1);
-        for (int o = 16; o > 0; o >>= 1) {
-            cnt_lo += __shfl_xor_sync(kFullMask, cnt_lo, o);
-            cnt_hi += __shfl_xor_sync(kFullMask, cnt_hi, o);
-        }
-        if (lane == 0) {
-            if (cnt_lo) atomicAdd(&hist[0], cnt_lo);
-            sh.w_hi[warp] = cnt_hi;
-        }
-        __syncthreads();
-        uint32_t cta_hi = 0;
-        for (int w = 0; w < kFusedWarps; ++w) cta_hi += sh.w_hi[w];
-        if (narrow) {
-            // publish this CTA's row: band bins and #key>hi
-            if (threadIdx.x < kRowWords) {
-                uint32_t v = 0;
-                if (threadIdx.x < kWarpBins) {
-                    for (int w = 0; w < kFusedWarps; ++w) v += sh.whist[w][threadIdx.x];
-                } else if (threadIdx.x == kWarpBins) {
-                    v = cta_hi;
+            if (narrow) {
+                // stream the run through the ring, one super-block ahead
+                if (!prefetched) issue_sb(sb0, 0);
+                int slot = 0;
+                auto count_sb = [&](int64_t sb, auto full_tag) {
+                    constexpr bool FULL = decltype(full_tag)::value;
+                    issue_sb(sb + 1, slot ^ 1);
+                    sb_wait();
+                    __syncwarp();   // the lane reads vectors that other lanes copied
+                    const uint32_t own = ring_own + slot * kSbBytes;
+                    uint32_t w[16];
+                    sb_read(own, rot, w);
+                    uint32_t hi_flags = 0, pending = 0;
+    #pragma unroll
+                    for (int g = 0; g < 4; ++g) {   // four words = eight elements at a time
+                        uint32_t a[4], b[4];
+    #pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t m = w[4 * g + i] & 0x7FFF7FFFu;
+                            a[i] = m + c_hi;                   // bit 15 of a half: key > hi
+                            b[i] = (m + c_lo) & ~a[i];         // bit 15 of a half: lo <= key <= hi
+                        }
+                        // above the band only the count matters: the flag bytes of all 16 words share one word
+                        hi_flags |= ((__byte_perm(a[0], a[1], 0x7531) & 0x80808080u) >> (2 * g)) |
+                                    ((__byte_perm(a[2], a[3], 0x7531) & 0x80808080u) >> (2 * g + 1));
+                        pending |= flags8(b[0], b[1], b[2], b[3]) << ((g ^ rot) << 3);
+                    }
+                    cnt_hi += __popc(hi_flags);
+                    if constexpr (!FULL) pending &= valid_mask32(sb * kSbElems + lane * 32, n);   // zero padding is no data
+                    while (pending) {   // a few percent of the elements: the band histogram (their order is irrelevant)
+                        const uint32_t e = top_bit(pending);
+                        pending ^= 1u << e;
+                        const uint32_t d = (lds_u16(own + 2u * e) & 0x7FFFu) - lo;
+                        if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
+                    }
+                    __syncwarp();   // every lane is done with the slot before it is refilled
+                    slot ^= 1;
+                };
+                int64_t sb = sb0;
+                for (; sb < sb_full_end; ++sb) count_sb(sb, std::true_type{});
+                for (; sb < sb1; ++sb) count_sb(sb, std::false_type{});
+                asm volatile("cp.async.wait_all;" ::: "memory");
+            } else {
+                int64_t blk = blk0;
+                for (; blk + kP1Blocks <= blk1; blk += kP1Blocks) {   // 4 loads per lane in flight
+                    uint4 va[kP1Blocks][kVpl];
+                    int na[kP1Blocks][kVpl];
+    #pragma unroll
+                    for (int u = 0; u < kP1Blocks; ++u) load_block(x, blk + u, lane, nvec_full, n, va[u], na[u]);
+    #pragma unroll
+                    for (int u = 0; u < kP1Blocks; ++u)
+    #pragma unroll
+                        for (int j = 0; j < kVpl; ++j) count_vec(va[u][j], na[u][j]);
                 }
-                rows[(size_t)blockIdx.x * kRowWords + threadIdx.x] = v;
+                for (; blk < blk1; ++blk) {
+                    uint4 va[kVpl];
+                    int na[kVpl];
+                    load_block(x, blk, lane, nvec_full, n, va, na);
+    #pragma unroll
+                    for (int j = 0; j < kVpl; ++j) count_vec(va[j], na[j]);
+                }
             }
-        } else {
-            // the global histogram is scratch that nobody cleared: every CTA clears a slice, and one more
-            // grid barrier separates the clearing from the accumulation
-            for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i <= width; i += gridDim.x * blockDim.x) ghist[i] = 0;
+            prefetched = false;
+            phase_stamp(st, 1);
+            for (int o = 16; o > 0; o >>= 1) {
+                cnt_lo += __shfl_xor_sync(kFullMask, cnt_lo, o);
+                cnt_hi += __shfl_xor_sync(kFullMask, cnt_hi, o);
+            }
+            if (lane == 0) {
+                if (cnt_lo) atomicAdd(&hist[0], cnt_lo);
+                sh.w_hi[warp] = cnt_hi;
+            }
+            __syncthreads();
+            uint32_t cta_hi = 0;
+            for (int w = 0; w < kFusedWarps; ++w) cta_hi += sh.w_hi[w];
+            if (narrow) {
+                // publish this CTA's row: band bins and #key>hi
+                if (threadIdx.x < kRowWords) {
+                    uint32_t v = 0;
+                    if (threadIdx.x < kWarpBins) {
+                        for (int w = 0; w < kFusedWarps; ++w) v += sh.whist[w][threadIdx.x];
+                    } else if (threadIdx.x == kWarpBins) {
+                        v = cta_hi;
+                    }
+                    rows[(size_t)blockIdx.x * kRowWords + threadIdx.x] = v;
+                }
+            } else {
+                // the global histogram is scratch that nobody cleared: every CTA clears a slice, and one more
+                // grid barrier separates the clearing from the accumulation
+                for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i <= width; i += gridDim.x * blockDim.x) ghist[i] = 0;
+                barrier_target += gridDim.x;
+                if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok, spin_max)) {
+                    if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
+                    return;
+                }
+                for (uint32_t i = threadIdx.x; i <= width; i += blockDim.x) {
+                    const uint32_t c = bins[i];
+                    if (c) atomicAdd(&ghist[i], c);
+                }
+                if (threadIdx.x == 0 && cta_hi) atomicAdd(&st->n_hi[attempt], (unsigned long long)cta_hi);
+            }
             barrier_target += gridDim.x;
             if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok, spin_max)) {
                 if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
                 return;
             }
-            for (uint32_t i = threadIdx.x; i <= width; i += blockDim.x) {
-                const uint32_t c = bins[i];
-                if (c) atomicAdd(&ghist[i], c);
-            }
-            if (threadIdx.x == 0 && cta_hi) atomicAdd(&st->n_hi[attempt], (unsigned long long)cta_hi);
-        }
-        barrier_target += gridDim.x;
-        if (!grid_barrier(&st->barrier, epoch, barrier_target, &sh.ok, spin_max)) {
-            if (threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
-            return;
         }
         phase_stamp(st, 2);
         if (threadIdx.x == 0) sh.found = 0;
@@ -964,9 +1015,9 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
 // ---------------------------------------------------------------------------------------------
 // Host side.
 // ---------------------------------------------------------------------------------------------
-dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool index32, void* values, void* meta,
-                                  uint32_t* offsets, void* workspace, size_t workspace_bytes, int32_t* dev_status,
-                                  cudaStream_t stream) {
+dropit_status fused_compress_bf16_prepared(const void* x, int64_t n, int64_t k, bool index32, void* values, void* meta,
+                                           uint32_t* offsets, void* workspace, size_t workspace_bytes,
+                                           int32_t* dev_status, cudaStream_t stream, const unsigned char* prep) {
     const FusedPlan plan = make_fused_plan(n);
     if (workspace_bytes < plan.total_bytes) return DROPIT_ERR_WORKSPACE;
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
@@ -989,13 +1040,230 @@ dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool inde
     uint32_t* maskp = index32 ? nullptr : reinterpret_cast<uint32_t*>(meta);
     int32_t* idxp = index32 ? reinterpret_cast<int32_t*>(meta) : nullptr;
     int spin_max = (int)spin_limit((uint32_t)kBarrierSpinLimit);
-    void* args[] = {&xp, &n, &kk, &bpw, &epoch, &ws, &h0, &h1, &ao, &ro, &vals, &maskp, &idxp, &offsets, &dev_status, &spin_max};
+    void* args[] = {&xp, &n, &kk, &bpw, &epoch, &ws, &h0, &h1, &ao, &ro, &vals, &maskp, &idxp, &offsets, &dev_status, &spin_max,
+                    &prep};
     const void* fn = index32 ? (const void*)fused_compress_kernel<true> : (const void*)fused_compress_kernel<false>;
     if (cudaLaunchCooperativeKernel(fn, dim3(plan.grid), dim3(kFusedThreads), args, index32 ? smem_idx : smem_mask,
                                     stream) != cudaSuccess) {
         cudaGetLastError();
         return DROPIT_ERR_CUDA;
     }
+    return check_launch();
+}
+
+dropit_status fused_compress_bf16(const void* x, int64_t n, int64_t k, bool index32, void* values, void* meta,
+                                  uint32_t* offsets, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                  cudaStream_t stream) {
+    return fused_compress_bf16_prepared(x, n, k, index32, values, meta, offsets, workspace, workspace_bytes, dev_status,
+                                        stream, nullptr);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The producer in front of the path: y = act(x) for a bf16 tensor that is about to become a conv / fc input
+// (Sec. 3.5: activations and normalisations keep their own caches; what they write is what DropIT compresses),
+// with the selection statistics of y taken on the way.  One read of x, one write of y; the selection kernel
+// then needs a single read of y.  Same work partition as fused_compress_kernel (a warp owns a run of
+// 1024-element super-blocks), same sample, same band, same per-warp histograms.
+// act: identity (y may be left out: statistics only), ReLU, or a table over all 65536 bf16 patterns
+// (any element-wise function; GELU is built by dropit_activation_table).  The table's entries for
+// 2^-9 <= |x| < 16 are kept in shared memory; the few elements outside that window read the table in
+// global memory.
+// ---------------------------------------------------------------------------------------------
+constexpr int kActIdentity = 0, kActRelu = 1, kActTable = 2;
+constexpr uint32_t kLutKeyLo = 118u << 7, kLutKeyHi = 131u << 7;   // keys of 2^-9 <= |x| < 2^4
+constexpr uint32_t kLutSpan = kLutKeyHi - kLutKeyLo;                // 1664 keys per sign
+constexpr size_t kLutBytes = 2 * kLutSpan * 2;
+
+template <int ACT>
+__device__ __forceinline__ uint32_t map_word(uint32_t w, uint32_t lut_addr, const uint16_t* __restrict__ table) {
+    if constexpr (ACT == kActIdentity) {
+        return w;
+    } else if constexpr (ACT == kActRelu) {
+        // max(x, 0): negative values and -0 become +0; NaN patterns (key > 0x7F80) pass
+        const uint32_t neg = w & kHiBits;
+        const uint32_t nan = ((w & 0x7FFF7FFFu) + 0x007F007Fu) & kHiBits;
+        const uint32_t kill = ((neg & ~nan) >> 15) * 0xFFFFu;
+        return w & ~kill;
+    } else {
+        const uint32_t i0 = (w & 0x7FFFu) - kLutKeyLo, i1 = ((w >> 16) & 0x7FFFu) - kLutKeyLo;
+        uint32_t y0, y1;
+        if (i0 < kLutSpan && i1 < kLutSpan) {
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(y0) : "r"(lut_addr + 2u * (((w >> 15) & 1u) * kLutSpan + i0)) : "memory");
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(y1) : "r"(lut_addr + 2u * ((w >> 31) * kLutSpan + i1)) : "memory");
+        } else {
+            y0 = __ldg(table + (w & 0xFFFFu));
+            y1 = __ldg(table + (w >> 16));
+        }
+        return y0 | (y1 << 16);
+    }
+}
+
+template <int ACT>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+produce_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t n, unsigned long long k, int blocks_per_warp,
+               const uint16_t* __restrict__ table, unsigned char* prep) {
+    extern __shared__ __align__(16) unsigned char fsm[];
+    uint32_t* sample_bins = reinterpret_cast<uint32_t*>(fsm + kRingBytes);
+    FusedShared& sh = *reinterpret_cast<FusedShared*>(fsm + kRingBytes + kStageBytes);
+    const uint32_t lut_addr = ptx_smem(fsm + kRingBytes + kStageBytes + ((sizeof(FusedShared) + 15) / 16) * 16);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring_warp = ptx_smem(fsm) + warp * (kRingSlots * kSbBytes);
+    const uint32_t ring_copy = ring_warp + lane * 16;
+    const uint32_t ring_own = ring_warp + lane * 64;
+    const uint32_t rot = (uint32_t)(lane >> 1) & 3u;
+    const int64_t nvec_full = n / 8;
+    const int64_t blocks_total = (n + kBlkElems - 1) / kBlkElems;
+    const int64_t blk0 = ((int64_t)blockIdx.x * kFusedWarps + warp) * blocks_per_warp;
+    int64_t blk1 = blk0 + blocks_per_warp;
+    if (blk1 > blocks_total) blk1 = blocks_total;
+    const int64_t sb0 = blk0 / 2, sb1 = (blk1 + 1) / 2;
+    const int64_t sb_full_end = (nvec_full / kSbVecs < sb1) ? nvec_full / kSbVecs : sb1;
+    if constexpr (ACT == kActTable) {
+        uint16_t* lut = reinterpret_cast<uint16_t*>(fsm + kRingBytes + kStageBytes + ((sizeof(FusedShared) + 15) / 16) * 16);
+        for (uint32_t i = threadIdx.x; i < 2 * kLutSpan; i += blockDim.x)
+            lut[i] = table[(i >= kLutSpan ? 0x8000u : 0u) | (kLutKeyLo + (i >= kLutSpan ? i - kLutSpan : i))];
+        __syncthreads();
+    }
+    auto map_vec = [&](const uint4& v) {
+        return make_uint4(map_word<ACT>(v.x, lut_addr, table), map_word<ACT>(v.y, lut_addr, table),
+                          map_word<ACT>(v.z, lut_addr, table), map_word<ACT>(v.w, lut_addr, table));
+    };
+    // the same sample as the selection kernel takes, seen through act: every CTA arrives at the same band
+    sample_band(x, n, k, sample_bins, sh.warp, sh.band, nullptr,
+                [&] { if (sb0 < sb_full_end) sb_issue_full(ring_copy, x + sb0 * kSbVecs + lane); }, map_vec);
+    const uint32_t lo = sh.band[0], hi = sh.band[1];
+    const uint32_t width = hi - lo;
+    const bool stats = n >= kSampleMinElems && width < (uint32_t)kWarpBins;   // uniform over the grid
+    for (int i = threadIdx.x; i < kFusedWarps * kWarpBins; i += blockDim.x) (&sh.whist[0][0])[i] = 0;
+    __syncthreads();
+    uint32_t* hist = sh.whist[warp];
+    const uint32_t c_hi = ge_const(hi + 1), c_lo = ge_const(lo);
+    uint32_t cnt_hi = 0, cnt_lo = 0;
+    // ---- whole super-blocks through the ring ----
+    {
+        int slot = 0;
+        for (int64_t sb = sb0; sb < sb_full_end; ++sb) {
+            if (sb + 1 < sb_full_end) sb_issue_full(ring_copy + (slot ^ 1) * kSbBytes, x + (sb + 1) * kSbVecs + lane);
+            else asm volatile("cp.async.commit_group;" ::: "memory");
+            sb_wait();
+            __syncwarp();
+            const uint32_t own = ring_own + slot * kSbBytes;
+            uint32_t w[16];
+            sb_read(own, rot, w);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w[i] = map_word<ACT>(w[i], lut_addr, table);
+            if (y != nullptr) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)   // registers 4j.. hold the lane's vector j ^ rot
+                    y[sb * kSbVecs + lane * 4 + (j ^ rot)] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            }
+            if (stats) {
+                if constexpr (ACT != kActIdentity) {   // the band walk below reads keys from the slot: they are y's now
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(own + ((j ^ rot) << 4)), "r"(w[4 * j]),
+                                     "r"(w[4 * j + 1]), "r"(w[4 * j + 2]), "r"(w[4 * j + 3]) : "memory");
+                }
+                uint32_t hi_flags = 0, pending = 0;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    uint32_t a[4], b[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t m = w[4 * g + i] & 0x7FFF7FFFu;
+                        a[i] = m + c_hi;                   // bit 15 of a half: key > hi
+                        b[i] = (m + c_lo) & ~a[i];         // bit 15 of a half: lo <= key <= hi
+                    }
+                    hi_flags |= ((__byte_perm(a[0], a[1], 0x7531) & 0x80808080u) >> (2 * g)) |
+                                ((__byte_perm(a[2], a[3], 0x7531) & 0x80808080u) >> (2 * g + 1));
+                    pending |= flags8(b[0], b[1], b[2], b[3]) << ((g ^ rot) << 3);
+                }
+                cnt_hi += __popc(hi_flags);
+                while (pending) {
+                    const uint32_t e = top_bit(pending);
+                    pending ^= 1u << e;
+                    const uint32_t d = (lds_u16(own + 2u * e) & 0x7FFFu) - lo;
+                    if (d == 0) ++cnt_lo; else atomicAdd(&hist[d], 1u);
+                }
+            }
+            __syncwarp();
+            slot ^= 1;
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+    }
+    // ---- the ragged last super-block of the tensor (at most one, in one warp): element by element ----
+    for (int64_t sb = (sb_full_end > sb0 ? sb_full_end : sb0); sb < sb1; ++sb) {
+        const uint16_t* xe = reinterpret_cast<const uint16_t*>(x);
+        uint16_t* ye = reinterpret_cast<uint16_t*>(y);
+        for (int i = 0; i < 32; ++i) {
+            const int64_t e = sb * kSbElems + lane * 32 + i;
+            if (e >= n) break;
+            const uint32_t xv = xe[e];
+            uint32_t yv;
+            if constexpr (ACT == kActTable) yv = __ldg(table + xv);
+            else yv = map_word<ACT>(xv, lut_addr, table) & 0xFFFFu;
+            if (ye != nullptr) ye[e] = (uint16_t)yv;
+            if (stats) {
+                const uint32_t key = yv & 0x7FFFu;
+                if (key > hi) ++cnt_hi;
+                else if (key >= lo) {
+                    if (key == lo) ++cnt_lo; else atomicAdd(&hist[key - lo], 1u);
+                }
+            }
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        cnt_lo += __shfl_xor_sync(kFullMask, cnt_lo, o);
+        cnt_hi += __shfl_xor_sync(kFullMask, cnt_hi, o);
+    }
+    if (lane == 0) {
+        if (cnt_lo) atomicAdd(&hist[0], cnt_lo);
+        sh.w_hi[warp] = cnt_hi;
+    }
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        PrepHeader* ph = reinterpret_cast<PrepHeader*>(prep);
+        ph->magic = kPrepMagic;
+        ph->valid = stats ? 1u : 0u;
+        ph->lo = lo;
+        ph->hi = hi;
+        ph->grid = gridDim.x;
+        ph->blocks_per_warp = (uint32_t)blocks_per_warp;
+        ph->n = (unsigned long long)n;
+        ph->k = k;
+    }
+    if (!stats) return;
+    uint32_t* rows = const_cast<uint32_t*>(prep_rows(prep));
+    uint32_t* wh = const_cast<uint32_t*>(prep_warp_hist(prep, gridDim.x)) + (size_t)blockIdx.x * kFusedWarps * kPrepWarpWords;
+    for (int i = threadIdx.x; i < kFusedWarps * kPrepWarpWords; i += blockDim.x) {
+        const int w = i / kPrepWarpWords, c = i % kPrepWarpWords;
+        wh[i] = c < kWarpBins ? sh.whist[w][c] : (c == kWarpBins ? sh.w_hi[w] : 0u);
+    }
+    if (threadIdx.x < kRowWords) {
+        uint32_t v = 0;
+        if (threadIdx.x < kWarpBins) {
+            for (int w = 0; w < kFusedWarps; ++w) v += sh.whist[w][threadIdx.x];
+        } else if (threadIdx.x == kWarpBins) {
+            for (int w = 0; w < kFusedWarps; ++w) v += sh.w_hi[w];
+        }
+        rows[(size_t)blockIdx.x * kRowWords + threadIdx.x] = v;
+    }
+}
+
+template <int ACT>
+static dropit_status launch_produce(const void* x, void* y, int64_t n, int64_t k, const uint16_t* table, unsigned char* prep,
+                                    cudaStream_t stream) {
+    const FusedPlan plan = make_fused_plan(n);
+    const size_t smem = kRingBytes + kStageBytes + ((sizeof(FusedShared) + 15) / 16) * 16 + kLutBytes;
+    static PerDeviceOnce attr;
+    if (attr.needed()) {
+        if (cudaFuncSetAttribute(produce_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return DROPIT_ERR_CUDA;
+        attr.mark();
+    }
+    produce_kernel<ACT><<<plan.grid, kFusedThreads, smem, stream>>>(reinterpret_cast<const uint4*>(x),
+                                                                    reinterpret_cast<uint4*>(y), n, (unsigned long long)k,
+                                                                    plan.blocks_per_warp, table, prep);
     return check_launch();
 }
 
@@ -1064,3 +1332,50 @@ extern "C" dropit_status dropit_compress_static(const void* x, int64_t n, double
                                kStaticScratchBytes, dev_status, stream);
 }
 
+
+extern "C" dropit_status dropit_produce_workspace(int64_t n, size_t* prep_bytes) {
+    if (n < 0 || n >= ((int64_t)1 << 31)) return DROPIT_ERR_INVALID_ARG;
+    if (prep_bytes) *prep_bytes = dropit::prep_bytes_for(n);
+    return DROPIT_OK;
+}
+
+extern "C" dropit_status dropit_produce(const void* x, int64_t n, double gamma, dropit_activation act, const uint16_t* table,
+                                        void* y, void* prep, size_t prep_bytes, void* cuda_stream) {
+    using namespace dropit;
+    if (n < 0 || n >= ((int64_t)1 << 31) || !(gamma >= 0.0 && gamma <= 1.0)) return DROPIT_ERR_INVALID_ARG;
+    if (act != DROPIT_ACT_IDENTITY && act != DROPIT_ACT_RELU && act != DROPIT_ACT_TABLE) return DROPIT_ERR_INVALID_ARG;
+    if (n == 0) return DROPIT_OK;
+    if (!x || !is_aligned16(x) || !prep || !is_aligned16(prep)) return DROPIT_ERR_INVALID_ARG;
+    if (y && (!is_aligned16(y) || y == x)) return DROPIT_ERR_INVALID_ARG;       // not in place: every CTA samples x
+    if (!y && act != DROPIT_ACT_IDENTITY) return DROPIT_ERR_INVALID_ARG;         // only the identity may leave y out
+    if (act == DROPIT_ACT_TABLE && (!table || !is_aligned16(table))) return DROPIT_ERR_INVALID_ARG;
+    if (prep_bytes < prep_bytes_for(n)) return DROPIT_ERR_WORKSPACE;
+    const int64_t k = dropit_keep_count(n, gamma);
+    cudaStream_t stream = as_stream(cuda_stream);
+    unsigned char* pp = reinterpret_cast<unsigned char*>(prep);
+    if (act == DROPIT_ACT_IDENTITY) return launch_produce<kActIdentity>(x, y, n, k, table, pp, stream);
+    if (act == DROPIT_ACT_RELU) return launch_produce<kActRelu>(x, y, n, k, table, pp, stream);
+    return launch_produce<kActTable>(x, y, n, k, table, pp, stream);
+}
+
+extern "C" dropit_status dropit_compress_prepared(const void* y, int64_t n, double gamma, dropit_format format,
+                                                  void* values, void* meta, uint32_t* offsets, const void* prep,
+                                                  size_t prep_bytes, void* workspace, size_t workspace_bytes,
+                                                  int32_t* dev_status, void* cuda_stream) {
+    using namespace dropit;
+    if (n < 0 || n >= ((int64_t)1 << 31) || !(gamma >= 0.0 && gamma <= 1.0)) return DROPIT_ERR_INVALID_ARG;
+    if (format != DROPIT_FMT_BITMASK && format != DROPIT_FMT_INDEX32) return DROPIT_ERR_INVALID_ARG;
+    if (n == 0) return DROPIT_OK;
+    if (!prep || !is_aligned16(prep)) return DROPIT_ERR_INVALID_ARG;
+    if (prep_bytes < prep_bytes_for(n)) return DROPIT_ERR_WORKSPACE;
+    const int64_t k = dropit_keep_count(n, gamma);
+    if (k == 0)   // nothing retained: the ordinary entry point zero-fills mask and table
+        return dropit_compress(y, n, gamma, DROPIT_BF16, format, values, meta, offsets, workspace, workspace_bytes,
+                               dev_status, cuda_stream);
+    if (!y || !offsets || !is_aligned16(y) || !is_aligned16(offsets)) return DROPIT_ERR_INVALID_ARG;
+    if (!meta || !is_aligned16(meta) || !values || !is_aligned16(values)) return DROPIT_ERR_INVALID_ARG;
+    if (!workspace || !is_aligned16(workspace)) return DROPIT_ERR_INVALID_ARG;
+    return fused_compress_bf16_prepared(y, n, k, format == DROPIT_FMT_INDEX32, values, meta, offsets, workspace,
+                                        workspace_bytes, dev_status, as_stream(cuda_stream),
+                                        reinterpret_cast<const unsigned char*>(prep));
+}
