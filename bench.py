@@ -14,7 +14,9 @@ on one GPU, the other named workloads (fp32 single Linear, ResNet-50 stage-1 con
 ViTDet-B linears at three drop ratios, the whole ViT-B/16 training step).
 The second form runs one entry point on one named workload a few times and prints each time:
 it is what the profiler command lines under profiles/ run.  OP is compress, compress_random,
-decompress, weight_grad or conv_weight_grad.
+decompress, weight_grad, conv_weight_grad, produce (the layer's activation fused with the selection
+statistics), compress_prepared (compression from those statistics) or torch_act (the stock
+activation kernel, for comparison).
 
 N > 1 is launched with torch.distributed.run, one rank per GPU; the path has no exchange step,
 so ranks are independent replicas (weak scaling) and NCCL only carries the barrier and the
@@ -194,15 +196,32 @@ class OpRunner:
         self.xs = [di.make_x(case, b).to(device) for b in range(nsets)]
         self.dys = [di.make_dy(case, b).to(device) for b in range(nsets)] if need_dy else None
         self.caches = [dropit.dropit_compress(x, case.gamma, fmt) for x in self.xs]
-        if op not in ("compress", "compress_random"):
+        self.act = {"gelu": "gelu", "relu": "relu"}.get(getattr(case, "x_dist", ""), "identity")
+        code = dropit.BF16 if case.dtype == "bf16" else dropit.F32
+        self.ws = torch.empty(max(dropit.dropit_cache_sizes(case.n, case.gamma, code, dropit.api._FMT_CODE[fmt])[3], 16),
+                              dtype=torch.uint8, device=device)
+        if op == "compress_prepared":   # statistics of the inputs themselves (taken by an identity producer)
+            self.preps = [dropit.dropit_produce(x, case.gamma, "identity", want_y=False)[1] for x in self.xs]
+        if op not in ("compress", "compress_random", "produce", "compress_prepared", "torch_act"):
             self.xs = None   # the dense inputs are not needed any more
 
     def __call__(self, i: int):
         d, c, b = self.dropit, self.case, i % self.nsets
         if self.op == "compress":
-            self.caches[b] = d.dropit_compress(self.xs[b], c.gamma, self.fmt)
+            self.caches[b] = d.dropit_compress(self.xs[b], c.gamma, self.fmt, workspace=self.ws)
         elif self.op == "compress_random":
             self.caches[b] = d.dropit_compress_random(self.xs[b], c.gamma, i, self.fmt)
+        elif self.op == "produce":            # the layer's activation (GELU / ReLU / copy) with the selection statistics
+            d.dropit_produce(self.xs[b], c.gamma, self.act)
+        elif self.op == "compress_prepared":
+            self.caches[b] = d.dropit_compress_prepared(self.xs[b], c.gamma, self.preps[b], self.fmt, workspace=self.ws)
+        elif self.op == "torch_act":          # the stock element-wise kernel that dropit_produce replaces
+            if self.act == "gelu":
+                torch.nn.functional.gelu(self.xs[b])
+            elif self.act == "relu":
+                torch.relu(self.xs[b])
+            else:
+                self.xs[b].clone()
         elif self.op == "decompress":
             d.dropit_decompress(self.caches[b])
         elif self.op == "weight_grad":
@@ -236,7 +255,9 @@ def run_only(args, device):
     run = OpRunner(op, case, device, args.format, 3 if args.queued else 1)
     if args.queued:
         us = run.queued_us(args.reps)
-        by = algorithmic_bytes_compress(case) if op.startswith("compress") else 0.0
+        by = algorithmic_bytes_compress(case) if op in ("compress", "compress_random") else (
+            compulsory_bytes_compress(case) if op == "compress_prepared" else (
+                2.0 * case.n * _elem_bytes(case) if op in ("produce", "torch_act") else 0.0))
         fl = dense_flops(case) if op.endswith("weight_grad") else 0.0
         rate = "%.0f GB/s algorithmic" % (by / us / 1e3) if by else ("%.0f TFLOP/s" % (fl / us / 1e6) if fl else "")
         print("%s %s gamma=%g %s: %.1f us per call over %d queued calls %s"
@@ -293,6 +314,26 @@ def other_workloads(device, peaks, reps: int = 20):
                           "conv_weight_grad": timed(di.R50_CONV1X1, "conv_weight_grad"), "bound": "hbm"}
     out["r50_conv3x3"] = {"compress": timed(di.R50_CONV3X3, "compress"),
                           "conv_weight_grad": timed(di.R50_CONV3X3, "conv_weight_grad"), "bound": "tensor"}
+    # the producer-fused path: the layer's activation with the selection statistics, then compression from them,
+    # beside the stock activation kernel followed by the ordinary compression
+    fused = {}
+    for case in (di.VITB_FC2, di.R50_CONV1X1, di.VITDET_FC2):
+        e = {}
+        for op in ("torch_act", "produce", "compress_prepared", "compress"):
+            run = OpRunner(op, case, device, "bitmask", 3)
+            e[op + "_us"] = run.queued_us(reps)
+            del run
+            torch.cuda.empty_cache()
+        io = 2.0 * case.n * _elem_bytes(case)
+        c = compulsory_bytes_compress(case)
+        e["produce_gbs"] = io / e["produce_us"] / 1e3
+        e["produce_frac_of_hbm_peak"] = e["produce_gbs"] / peaks["hbm_gbs"]
+        e["compress_prepared_gbs"] = c / e["compress_prepared_us"] / 1e3          # one read of y + the outputs
+        e["compress_prepared_frac_of_hbm_peak"] = e["compress_prepared_gbs"] / peaks["hbm_gbs"]
+        e["stock_pair_us"] = e["torch_act_us"] + e["compress_us"]
+        e["fused_pair_us"] = e["produce_us"] + e["compress_prepared_us"]
+        fused[case.name] = e
+    out["producer_fused"] = fused
     # configuration 4: ViTDet-B linears at three drop ratios
     for base in (di.VITDET_QKV, di.VITDET_FC1, di.VITDET_FC2):
         for g in (0.5, 0.8, 0.9):
@@ -305,13 +346,14 @@ def vit_step(device, batch: int = 64, gamma: float = 0.9, steps: int = 5):
     """Configuration 5: the whole ViT-B/16 training step, stock layers against DropIT on every Linear."""
     from paper_2202_13808_b200 import vit
     res = {}
-    for name, g in (("dense", None), ("dropit", gamma)):
-        model = vit.build_vit_b16(g, device=device)
+    for name, g, fuse in (("dense", None, False), ("dropit", gamma, False), ("dropit_fused_gelu", gamma, True)):
+        model = vit.build_vit_b16(g, device=device, fuse_gelu=fuse)
         sps, peak, loss = vit.train_steps(model, batch, steps)
         res[name] = {"samples_per_s": sps, "peak_step_bytes": peak, "loss": loss}
         del model
         torch.cuda.empty_cache()
     res["speed_ratio"] = res["dropit"]["samples_per_s"] / res["dense"]["samples_per_s"]
+    res["speed_ratio_fused_gelu"] = res["dropit_fused_gelu"]["samples_per_s"] / res["dense"]["samples_per_s"]
     res["peak_ratio"] = res["dropit"]["peak_step_bytes"] / max(res["dense"]["peak_step_bytes"], 1)
     res["config"] = {"model": "ViT-B/16", "depth": 12, "batch": batch, "gamma": gamma, "dtype": "bf16", "steps": steps}
     return res

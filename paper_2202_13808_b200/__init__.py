@@ -12,4 +12,6 @@ from .api import (  # noqa: F401
     dropit_weight_grad_workspace, check_device_status, library_path,
     dropit_activation_table, dropit_produce, dropit_produce_workspace, dropit_compress_prepared,
 )
-from .nn import DropITConv2d, DropITConv2dFn, DropITLinear, DropITLinearFn, convert_linear_layers  # noqa: F401
+from .nn import (  # noqa: F401
+    DropITConv2d, DropITConv2dFn, DropITGeluLinear, DropITGeluLinearFn, DropITLinear, DropITLinearFn, convert_linear_layers,
+)

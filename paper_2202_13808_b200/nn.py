@@ -28,6 +28,15 @@ def _compress(x: torch.Tensor, gamma: float, fmt: str, seed):
     return api.dropit_compress_random(x, gamma, int(seed), fmt)
 
 
+def _cache_dtype(x: torch.Tensor, weight: torch.Tensor) -> torch.dtype:
+    """The dtype the layer's matmul really runs in, which is the dtype its input is cached in: under autocast
+    the autocast dtype, otherwise the weight's.  (An fp32 activation in front of bf16 weights would otherwise be
+    cached in fp32 and take the fp32 kernels, three times the cache and no tensor cores.)  Anything but bf16
+    falls back to the input's own dtype."""
+    dt = torch.get_autocast_dtype("cuda") if torch.is_autocast_enabled("cuda") else weight.dtype
+    return torch.bfloat16 if dt == torch.bfloat16 else x.dtype
+
+
 def _check_input(x: torch.Tensor):
     if not x.is_cuda:
         raise ValueError("DropIT layers need CUDA tensors (there is no CPU path)")
@@ -43,10 +52,13 @@ class DropITLinearFn(torch.autograd.Function):
         _check_input(x)
         z = F.linear(x, weight, bias)
         ctx.has_bias = bias is not None
-        ctx.x_shape = tuple(x.shape)
+        ctx.bias_dtype = bias.dtype if bias is not None else None
+        ctx.x_shape, ctx.x_dtype = tuple(x.shape), x.dtype
         ctx.cache_meta = None
         if weight.requires_grad:
             x2 = x.reshape(-1, x.shape[-1])
+            if x2.dtype != _cache_dtype(x2, weight):
+                x2 = x2.to(torch.bfloat16)
             if not x2.is_contiguous():
                 x2 = x2.contiguous()
             cache = _compress(x2, gamma, fmt, seed)
@@ -63,7 +75,7 @@ class DropITLinearFn(torch.autograd.Function):
         dx = dw = db = None
         dz2 = dz.reshape(-1, dz.shape[-1])
         if ctx.needs_input_grad[0]:
-            dx = (dz2 @ weight).reshape(ctx.x_shape)          # Eq. 3: exact, needs theta only
+            dx = (dz2 @ weight.to(dz2.dtype)).reshape(ctx.x_shape).to(ctx.x_dtype)   # Eq. 3: exact, needs theta only
         if ctx.needs_input_grad[1] and ctx.cache_meta is not None:
             n, k, shape, dtype, fmt, gamma = ctx.cache_meta
             cache = api.DropITCache(saved[1], saved[2], saved[3], n, k, shape, dtype, fmt, gamma)
@@ -72,7 +84,7 @@ class DropITLinearFn(torch.autograd.Function):
                 dzc = dzc.to(dtype)
             dw = api.dropit_weight_grad(dzc, cache).to(weight.dtype)   # Eq. 6
         if ctx.has_bias and ctx.needs_input_grad[2]:
-            db = dz2.sum(0)
+            db = dz2.sum(0).to(ctx.bias_dtype)
         return dx, dw, db, None, None, None
 
 
@@ -88,7 +100,8 @@ class DropITConv2dFn(torch.autograd.Function):
         ctx.stride, ctx.padding = stride, padding
         ctx.cache_meta = None
         if weight.requires_grad:
-            xc = x if x.is_contiguous() else x.contiguous()
+            xc = x if x.dtype == _cache_dtype(x, weight) else x.to(torch.bfloat16)
+            xc = xc if xc.is_contiguous() else xc.contiguous()
             cache = _compress(xc, gamma, fmt, seed)
             ctx.cache_meta = (cache.n, cache.k, cache.shape, cache.dtype, cache.fmt, cache.gamma)
             ctx.save_for_backward(weight, cache.values, cache.meta, cache.offsets)
@@ -114,6 +127,43 @@ class DropITConv2dFn(torch.autograd.Function):
         if ctx.has_bias and ctx.needs_input_grad[2]:
             db = dz.sum((0, 2, 3))
         return dx, dw, db, None, None, None, None, None
+
+
+class DropITGeluLinearFn(torch.autograd.Function):
+    """z = GELU(x) W^T + b for bf16 tensors, with the GELU written by the library's producer kernel so that the
+    selection statistics of GELU(x), the tensor the Linear caches, are taken while it is written (Sec. 3.5: the
+    activation keeps its own cache x; only the Linear's cache is replaced by D(GELU(x)))."""
+
+    @staticmethod
+    def forward(ctx, x, weight, bias, gamma: float, fmt: str):
+        _check_input(x)
+        x2 = x.reshape(-1, x.shape[-1])
+        x2 = x2 if x2.is_contiguous() else x2.contiguous()
+        y, prep = api.dropit_produce(x2, gamma, "gelu")
+        z = F.linear(y, weight, bias).reshape(*x.shape[:-1], weight.shape[0])
+        ctx.has_bias = bias is not None
+        ctx.x_shape = tuple(x.shape)
+        cache = api.dropit_compress_prepared(y, gamma, prep, fmt)
+        ctx.cache_meta = (cache.n, cache.k, cache.shape, cache.dtype, cache.fmt, cache.gamma)
+        ctx.save_for_backward(x2, weight, cache.values, cache.meta, cache.offsets)
+        return z
+
+    @staticmethod
+    def backward(ctx, dz):
+        x2, weight, values, meta, offsets = ctx.saved_tensors
+        dx = dw = db = None
+        dz2 = dz.reshape(-1, dz.shape[-1])
+        if ctx.needs_input_grad[0]:
+            dy = dz2 @ weight                                             # Eq. 3: exact, needs theta only
+            dx = torch.ops.aten.gelu_backward(dy, x2).reshape(ctx.x_shape)   # the activation's own cache is x
+        if ctx.needs_input_grad[1]:
+            n, k, shape, dtype, fmt, gamma = ctx.cache_meta
+            cache = api.DropITCache(values, meta, offsets, n, k, shape, dtype, fmt, gamma)
+            dzc = dz2 if dz2.is_contiguous() else dz2.contiguous()
+            dw = api.dropit_weight_grad(dzc.to(dtype), cache).to(weight.dtype)   # Eq. 6
+        if ctx.has_bias and ctx.needs_input_grad[2]:
+            db = dz2.sum(0)
+        return dx, dw, db, None, None
 
 
 class _Strategy:
@@ -146,6 +196,20 @@ class DropITLinear(nn.Linear, _Strategy):
         return DropITLinearFn.apply(x, self.weight, self.bias, self.gamma, self.fmt, self._next_seed())
 
 
+class DropITGeluLinear(nn.Linear):
+    """GELU followed by nn.Linear (an MLP's second layer together with the activation in front of it), bf16, with the
+    Linear's input cache compressed from statistics that the GELU kernel takes on the way."""
+
+    def __init__(self, in_features, out_features, bias=True, gamma: float = 0.9, fmt: str = "bitmask", **kw):
+        super().__init__(in_features, out_features, bias=bias, **kw)
+        self.gamma, self.fmt = float(gamma), fmt
+
+    def forward(self, x):
+        if not (self.training and torch.is_grad_enabled()) or x.dtype != torch.bfloat16:
+            return F.linear(F.gelu(x), self.weight, self.bias)
+        return DropITGeluLinearFn.apply(x, self.weight, self.bias, self.gamma, self.fmt)
+
+
 class DropITConv2d(nn.Conv2d, _Strategy):
     """nn.Conv2d (groups 1, dilation 1, square stride/padding) with a compressed input cache."""
 
@@ -169,7 +233,7 @@ def convert_linear_layers(module: nn.Module, gamma: float, fmt: str = "bitmask",
     """Replace every nn.Linear below `module` (except names in `skip`) by a DropITLinear sharing its parameters."""
     skip = skip or set()
     for name, child in list(module.named_children()):
-        if isinstance(child, nn.Linear) and not isinstance(child, DropITLinear) and name not in skip:
+        if isinstance(child, nn.Linear) and not isinstance(child, (DropITLinear, DropITGeluLinear)) and name not in skip:
             new = DropITLinear(child.in_features, child.out_features, bias=child.bias is not None, gamma=gamma, fmt=fmt,
                                device=child.weight.device, dtype=child.weight.dtype)
             new.weight, new.bias = child.weight, child.bias

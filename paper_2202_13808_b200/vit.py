@@ -17,7 +17,7 @@ import torch
 import torch.nn as nn
 import torch.nn.functional as F
 
-from .nn import convert_linear_layers
+from .nn import DropITGeluLinear, convert_linear_layers
 
 
 class Block(nn.Module):
@@ -30,13 +30,15 @@ class Block(nn.Module):
         self.norm2 = nn.LayerNorm(dim)
         self.fc1 = nn.Linear(dim, mlp)
         self.fc2 = nn.Linear(mlp, dim)
+        self.gelu_in_fc2 = False      # True when fc2 is a DropITGeluLinear, which applies the GELU itself
 
     def forward(self, x):
         B, L, C = x.shape
         qkv = self.qkv(self.norm1(x)).reshape(B, L, 3, self.heads, C // self.heads).permute(2, 0, 3, 1, 4)
         a = F.scaled_dot_product_attention(qkv[0], qkv[1], qkv[2])
         x = x + self.proj(a.transpose(1, 2).reshape(B, L, C))
-        return x + self.fc2(F.gelu(self.fc1(self.norm2(x))))
+        h = self.fc1(self.norm2(x))
+        return x + (self.fc2(h) if self.gelu_in_fc2 else self.fc2(F.gelu(h)))
 
 
 class ViT(nn.Module):
@@ -58,11 +60,20 @@ class ViT(nn.Module):
         return self.head(self.norm(x)[:, 0])
 
 
-def build_vit_b16(gamma=None, device="cuda", dtype=torch.bfloat16, depth=12, seed=0) -> ViT:
-    """Random-initialised ViT-B/16; gamma=None keeps stock layers, otherwise every nn.Linear becomes DropITLinear."""
+def build_vit_b16(gamma=None, device="cuda", dtype=torch.bfloat16, depth=12, seed=0, fuse_gelu=False) -> ViT:
+    """Random-initialised ViT-B/16; gamma=None keeps stock layers, otherwise every nn.Linear becomes DropITLinear.
+    fuse_gelu: the MLP's GELU and second Linear become one DropITGeluLinear (the GELU kernel takes the selection
+    statistics of its output, the compression reads that output once)."""
     torch.manual_seed(seed)
     model = ViT(depth=depth).to(device=device, dtype=dtype)
     if gamma is not None:
+        if fuse_gelu:
+            for b in model.blocks:
+                old = b.fc2
+                new = DropITGeluLinear(old.in_features, old.out_features, gamma=gamma, device=old.weight.device,
+                                       dtype=old.weight.dtype)
+                new.weight, new.bias = old.weight, old.bias
+                b.fc2, b.gelu_in_fc2 = new, True
         convert_linear_layers(model, gamma)
     return model.train()
 

@@ -117,3 +117,78 @@ def test_vit_step_runs_with_dropit_on_every_linear(cuda_device):
     sps, peak, loss = train_steps(model, batch=8, steps=2, warmup=1)
     assert sps > 0 and np.isfinite(loss)
     dropit.check_device_status(cuda_device)
+
+
+def test_gelu_linear_module_uses_the_producer_and_matches_the_oracle(cuda_device):
+    """GELU + Linear with the GELU written by dropit_produce: the forward is the correctly rounded GELU followed by
+    the stock matmul, the weight gradient is Eq. 6 on the min-k cache of GELU(x), the input gradient goes through
+    the activation's own (dense) cache."""
+    from paper_2202_13808_b200.nn import DropITGeluLinear
+    torch.manual_seed(3)
+    M, Ca, Cz = 1024, 768, 256                       # 786 432 elements: large enough for the sampled path
+    x = torch.randn(M, Ca, device=cuda_device).to(torch.bfloat16).requires_grad_(True)
+    dz = (torch.randn(M, Cz, device=cuda_device) * 0.02).to(torch.bfloat16)
+    lin = DropITGeluLinear(Ca, Cz, gamma=0.9, device=cuda_device, dtype=torch.bfloat16).train()
+    z = lin(x)
+    z.backward(dz)
+    # forward: table GELU (rounded once from double) then F.linear
+    xb = x.detach().cpu().view(torch.int16).numpy().view(np.uint16).reshape(-1)
+    yb = oracle.apply_table(oracle.activation_table(oracle.ACT_GELU), xb)
+    y = torch.from_numpy(yb.view(np.int16)).view(torch.bfloat16).reshape(M, Ca).to(cuda_device)
+    assert torch.equal(z, F.linear(y, lin.weight, lin.bias))
+    # weight gradient: the oracle's Eq. 6 on min-k of GELU(x)
+    keep, k = oracle.min_k(yb, 0.9, oracle.BF16)
+    dzb, _ = oracle.to_bits(dz.cpu())
+    dw = oracle.fc_weight_grad(dzb, yb, keep, M, Ca, Cz, oracle.BF16)
+    assert max_rel_err(lin.weight.grad.float().cpu().numpy(), dw) < 1e-2
+    # input gradient: stock GELU backward of dz W
+    x2 = x.detach().clone().requires_grad_(True)
+    F.linear(F.gelu(x2), lin.weight, lin.bias).backward(dz)
+    assert torch.allclose(x.grad.float(), x2.grad.float(), rtol=2e-2, atol=1e-4)
+    dropit.check_device_status(cuda_device)
+
+
+def test_fp32_activation_in_front_of_bf16_weights_is_cached_in_bf16(cuda_device):
+    """Under autocast (or with fp32 activations and bf16 weights) the matmul runs in bf16, so the cache is bf16:
+    a third of the bytes of an fp32 cache, and the tensor-core weight gradient."""
+    torch.manual_seed(4)
+    lin = DropITLinear(256, 128, gamma=0.9, device=cuda_device, dtype=torch.float32).train()
+    x = torch.randn(4096, 256, device=cuda_device, requires_grad=True)
+    saved = []
+    with torch.autograd.graph.saved_tensors_hooks(lambda t: (saved.append(t), t)[1], lambda t: t):
+        with torch.autocast("cuda", dtype=torch.bfloat16):
+            z = lin(x)
+    assert z.dtype == torch.bfloat16
+    assert any(t.dtype == torch.bfloat16 and t.numel() == dropit.dropit_keep_count(x.numel(), 0.9) for t in saved)
+    z.float().sum().backward()
+    assert lin.weight.grad is not None and torch.isfinite(lin.weight.grad).all()
+    dropit.check_device_status(cuda_device)
+
+
+def test_vit_step_with_the_gelu_fused_into_fc2(cuda_device):
+    from paper_2202_13808_b200.nn import DropITGeluLinear
+    from paper_2202_13808_b200.vit import build_vit_b16, train_steps
+    model = build_vit_b16(0.9, device=cuda_device, depth=2, fuse_gelu=True)
+    assert sum(isinstance(m, DropITGeluLinear) for m in model.modules()) == 2
+    assert sum(isinstance(m, DropITLinear) for m in model.modules()) == 2 * 3 + 1
+    sps, peak, loss = train_steps(model, batch=8, steps=2, warmup=1)
+    assert sps > 0 and np.isfinite(loss)
+    dropit.check_device_status(cuda_device)
+
+
+@pytest.mark.skipif(torch.cuda.device_count() < 2, reason="needs two visible devices")
+def test_second_device_in_the_same_process():
+    """Kernel attributes and cached plans are kept per device: after cuda:0 has been used, cuda:1 compresses and
+    takes a weight gradient in the same process (each GPU works on its own memory only; no peer access)."""
+    case = di.small_linear(640, 768, 384, "bf16", 0.9)
+    x, dy = di.make_x(case), di.make_dy(case)
+    bits, dt, keep, k = oracle_cache(x, case.gamma)
+    dyb, _ = oracle.to_bits(dy)
+    ref = oracle.fc_weight_grad(dyb, bits, keep, case.M, case.Ca, case.Cz, dt)
+    for dev in (torch.device("cuda:0"), torch.device("cuda:1")):
+        cache = dropit.dropit_compress(x.to(dev), case.gamma, "bitmask")
+        dw = dropit.dropit_weight_grad(dy.to(dev), cache)
+        dwf = dropit.dropit_weight_grad(dy.to(dev), cache, fused=True)
+        dropit.check_device_status(dev)
+        assert cache.k == k
+        assert max_rel_err(dw.cpu().numpy(), ref) < 2e-4 and max_rel_err(dwf.cpu().numpy(), ref) < 2e-4
