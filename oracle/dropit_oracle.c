@@ -23,6 +23,10 @@
  *                          tensor stated as a table over all 65536 bit patterns (act evaluated in double,
  *                          rounded once to bf16, ties to even), and the histogram of the ordering keys of y
  *
+ *   - 8-bit retained values   Sec. 1 / Table 5 combine DropIT with 8-bit and 4-bit activation quantisers on the
+ *                          other layers; here the same idea on DropIT's own payload: the retained bf16 values
+ *                          as sign + 3 exponent bits + 4 mantissa bits under one exponent shared by the tensor
+ *
  * Floating point: products and sums in double; results are returned as double.
  * Elements are passed as raw bits (uint16 for bf16, uint32 for fp32); the
  * ordering key of an element is its bits with the sign bit cleared, so
@@ -415,6 +419,61 @@ void oracle_apply_table(const uint16_t* table, const uint16_t* x, int64_t n, uin
 void oracle_key_histogram_bf16(const uint16_t* x, int64_t n, uint64_t* hist /* 32768 */) {
     memset(hist, 0, 32768 * sizeof(uint64_t));
     for (int64_t i = 0; i < n; ++i) hist[x[i] & 0x7FFF] += 1;
+}
+
+/* ---- retained values in 8 bits ------------------------------------------- */
+
+/* Min-k retains the LARGEST magnitudes, so the retained values of a tensor span few binades: eight bits hold
+ * them well.  The code is a small floating-point number, sign | e (3 bits) | m (4 bits), scaled by the tensor's
+ * top exponent field E_top (the largest exponent field among its finite retained values):
+ *     u = 2^(E_top - 127 - 10)                    one step of the lowest binade
+ *     e = 0:       value = m * u                  (zero and the sub-binade below 16 u)
+ *     e = 1 .. 7:  value = (16 + m) * 2^(e-1) * u (the top binade, e = 7, is the binade of E_top)
+ * A value is rounded to the nearest code, ties to even (in code order); above the largest code it saturates,
+ * and so do Inf and NaN patterns.  With E_top < 11 (everything below 2^-116) every code is zero.
+ * |decode(encode(v)) - v| <= |v| / 32 for 16 u <= |v| <= the largest code, and <= u / 2 below. */
+uint32_t oracle_q8_top_exponent(const uint16_t* values, int64_t k) {
+    uint32_t top = 0;
+    for (int64_t i = 0; i < k; ++i) {
+        const uint32_t e = (values[i] >> 7) & 0xFFu;
+        if (e != 0xFFu && e > top) top = e;
+    }
+    return top;
+}
+
+uint8_t oracle_q8_encode_one(uint16_t v, uint32_t e_top) {
+    const uint8_t sign = (uint8_t)((v >> 8) & 0x80u);
+    if (((v >> 7) & 0xFFu) == 0xFFu) return (uint8_t)(sign | 0x7Fu);
+    if (e_top < 11) return sign;
+    const double a = ldexp(fabs(bf16_bits_to_double(v)), 127 + 10 - (int)e_top);   /* |v| / u, exact */
+    double code;
+    if (a < 16.0) {
+        code = rint(a);                                   /* 0 .. 16 (16 is the first code of e = 1) */
+    } else {
+        int ex;
+        (void)frexp(a, &ex);                              /* a in [2^(ex-1), 2^ex): binade e = ex - 4 */
+        const int e = ex - 4;
+        code = (double)((e - 1) << 4) + rint(ldexp(a, -(e - 1)));   /* mantissa in 16 .. 32; 32 carries into e + 1 */
+    }
+    if (code > 127.0) code = 127.0;
+    return (uint8_t)(sign | (uint8_t)code);
+}
+
+uint16_t oracle_q8_decode_one(uint8_t q, uint32_t e_top) {
+    const uint16_t sign = (uint16_t)((q & 0x80u) << 8);
+    const uint32_t c = q & 0x7Fu;
+    if (c == 0 || e_top < 11) return sign;
+    const uint32_t e = c >> 4, m = c & 15u;
+    const double val = (e == 0) ? ldexp((double)m, (int)e_top - 137) : ldexp((double)(16 + m), (int)e_top - 137 + (int)e - 1);
+    return (uint16_t)(sign | oracle_round_to_bf16(val));  /* exact: at most five significant bits */
+}
+
+void oracle_q8_encode(const uint16_t* values, int64_t k, uint32_t e_top, uint8_t* codes) {
+    for (int64_t i = 0; i < k; ++i) codes[i] = oracle_q8_encode_one(values[i], e_top);
+}
+
+void oracle_q8_decode(const uint8_t* codes, int64_t k, uint32_t e_top, uint16_t* values) {
+    for (int64_t i = 0; i < k; ++i) values[i] = oracle_q8_decode_one(codes[i], e_top);
 }
 
 int oracle_num_threads(void) {

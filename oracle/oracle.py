@@ -19,6 +19,7 @@ __all__ = [
     "recover_from_index32", "fc_weight_grad", "fc_weight_grad_entries", "conv_weight_grad",
     "conv_weight_grad_entries", "num_threads", "bits_to_float64", "philox4x32_10", "random_ranks", "random_k",
     "ACT_IDENTITY", "ACT_RELU", "ACT_GELU", "round_to_bf16", "activation_table", "apply_table", "key_histogram_bf16",
+    "q8_top_exponent", "q8_encode", "q8_decode",
 ]
 
 BF16 = 0
@@ -55,6 +56,7 @@ def _load():
             lib.oracle_min_k.restype = ctypes.c_int
             lib.oracle_random_k.restype = ctypes.c_int
             lib.oracle_num_threads.restype = ctypes.c_int
+            lib.oracle_q8_top_exponent.restype = ctypes.c_uint32
             lib.oracle_round_to_bf16.restype = ctypes.c_uint16
             lib.oracle_round_to_bf16.argtypes = [ctypes.c_double]
             _lib = lib
@@ -307,3 +309,26 @@ def key_histogram_bf16(x_bits: np.ndarray) -> np.ndarray:
     hist = np.zeros(32768, np.uint64)
     _load().oracle_key_histogram_bf16(_p(x), _i64(x.size), _p(hist))
     return hist
+
+
+def q8_top_exponent(values_bits: np.ndarray) -> int:
+    """Largest exponent field among the finite values: the scale of the tensor's 8-bit codes."""
+    v = _check_bits(values_bits, BF16)
+    return int(_load().oracle_q8_top_exponent(_p(v), _i64(v.size)))
+
+
+def q8_encode(values_bits: np.ndarray, e_top: int) -> np.ndarray:
+    """Retained bf16 values as 8-bit codes sign | e3 | m4 under the shared top exponent (Sec. 1, Table 5: DropIT
+    combined with 8-bit quantisation, here on DropIT's own payload)."""
+    v = _check_bits(values_bits, BF16)
+    out = np.empty(v.size, np.uint8)
+    _load().oracle_q8_encode(_p(v), _i64(v.size), ctypes.c_uint32(int(e_top)), _p(out))
+    return out
+
+
+def q8_decode(codes: np.ndarray, e_top: int) -> np.ndarray:
+    """The bf16 values that the 8-bit codes stand for."""
+    c = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty(c.size, np.uint16)
+    _load().oracle_q8_decode(_p(c), _i64(c.size), ctypes.c_uint32(int(e_top)), _p(out))
+    return out
