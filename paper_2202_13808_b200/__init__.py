@@ -11,6 +11,7 @@ from .api import (  # noqa: F401
     dropit_decompress, dropit_keep_count, dropit_launch_count, dropit_status_string, dropit_version, dropit_weight_grad,
     dropit_weight_grad_workspace, check_device_status, library_path,
     dropit_activation_table, dropit_produce, dropit_produce_workspace, dropit_compress_prepared,
+    dropit_quantize_cache, dropit_dequantize_cache,
 )
 from .nn import (  # noqa: F401
     DropITConv2d, DropITConv2dFn, DropITGeluLinear, DropITGeluLinearFn, DropITLinear, DropITLinearFn, convert_linear_layers,

@@ -25,6 +25,8 @@ SIGNATURES = {
     "dropit_compress_random_workspace": (c_int, [c_i64, c_dbl, p_sz]),
     "dropit_compress_random": (c_int, [c_vp, c_i64, c_dbl, ctypes.c_uint64, c_int, c_int, c_vp, c_vp, c_vp, c_vp, c_sz,
                                        c_vp, c_vp]),
+    "dropit_quantize_values": (c_int, [c_vp, c_i64, c_vp, c_vp, c_vp]),
+    "dropit_dequantize_values": (c_int, [c_vp, c_vp, c_i64, c_vp, c_vp]),
     "dropit_activation_table": (c_int, [c_int, c_vp, c_vp]),
     "dropit_produce_workspace": (c_int, [c_i64, p_sz]),
     "dropit_produce": (c_int, [c_vp, c_i64, c_dbl, c_int, c_vp, c_vp, c_vp, c_sz, c_vp]),

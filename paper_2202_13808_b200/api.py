@@ -79,9 +79,13 @@ class DropITCache:
     fmt: int
     gamma: float
 
+    codes: Optional[torch.Tensor] = None    # 8-bit codes of the values (dropit_quantize_cache); then `values` is None
+    scale: Optional[torch.Tensor] = None    # the codes' shared top exponent (one int32 on the device)
+
     @property
     def nbytes(self) -> int:
-        return sum(t.numel() * t.element_size() for t in (self.values, self.meta, self.offsets))
+        parts = (self.values, self.meta, self.offsets, self.codes, self.scale)
+        return sum(t.numel() * t.element_size() for t in parts if t is not None)
 
 
 _status_words = {}
@@ -148,6 +152,36 @@ def dropit_compress(x: torch.Tensor, gamma: float, fmt="bitmask", workspace: Opt
                                    _ptr(workspace), workspace.numel(), _ptr(_status_word(dev)), _stream_ptr(dev))
     _check(code, "dropit_compress")
     return DropITCache(values, meta, offsets, n, k, tuple(x.shape), x.dtype, fmt, float(gamma))
+
+
+def dropit_quantize_cache(cache: DropITCache) -> DropITCache:
+    """The same cache with its bf16 values replaced by 8-bit codes (sign, 3 exponent bits, 4 mantissa bits under the
+    tensor's top exponent): 1 byte per retained element.  Mask / indices and seek table are shared with `cache`."""
+    if cache.dtype != torch.bfloat16:
+        raise TypeError("8-bit codes are defined for bf16 caches")
+    if cache.values is None:
+        return cache
+    dev = cache.values.device if cache.k else cache.offsets.device
+    codes = torch.empty(cache.k, dtype=torch.uint8, device=dev)
+    scale = torch.zeros(1, dtype=torch.int32, device=dev)
+    with _on_device(dev):
+        code = _lib.load().dropit_quantize_values(_ptr(cache.values), cache.k, _ptr(codes), _ptr(scale), _stream_ptr(dev))
+    _check(code, "dropit_quantize_values")
+    return DropITCache(None, cache.meta, cache.offsets, cache.n, cache.k, cache.shape, cache.dtype, cache.fmt,
+                       cache.gamma, codes, scale)
+
+
+def dropit_dequantize_cache(cache: DropITCache) -> DropITCache:
+    """A cache with bf16 values again (exactly the values the codes stand for); a no-op for an unquantised cache."""
+    if cache.values is not None:
+        return cache
+    dev = cache.scale.device
+    values = torch.empty(cache.k, dtype=torch.bfloat16, device=dev)
+    with _on_device(dev):
+        code = _lib.load().dropit_dequantize_values(_ptr(cache.codes), _ptr(cache.scale), cache.k, _ptr(values),
+                                                    _stream_ptr(dev))
+    _check(code, "dropit_dequantize_values")
+    return DropITCache(values, cache.meta, cache.offsets, cache.n, cache.k, cache.shape, cache.dtype, cache.fmt, cache.gamma)
 
 
 ACT_IDENTITY, ACT_RELU, ACT_TABLE = 0, 1, 2
@@ -265,6 +299,7 @@ def dropit_compress_random(x: torch.Tensor, gamma: float, seed: int, fmt="bitmas
 
 def dropit_decompress(cache: DropITCache, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """R(a-hat) (Sec. 3.2): dense tensor, dropped positions +0; written into `out` when given."""
+    cache = dropit_dequantize_cache(cache)
     lib = _lib.load()
     dev = cache.offsets.device if cache.offsets.numel() else cache.values.device
     if out is None:
@@ -305,6 +340,7 @@ def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch
     """Eq. 6: dW[j, c] = sum over retained (n, c) of dY[n, j] a[n, c]; returns fp32 [Cz, Ca].
 
     fused=True calls dropit_weight_grad_fused (cache expanded inside the GEMM, no dense scratch)."""
+    cache = dropit_dequantize_cache(cache)
     _require_cuda(dy, "dy")
     if dy.dtype != cache.dtype:
         raise TypeError("dy dtype %s != cache dtype %s" % (dy.dtype, cache.dtype))
@@ -351,6 +387,7 @@ def dropit_conv_weight_grad(dy: torch.Tensor, cache: DropITCache, kernel_size: T
                             pad: int = 0, dilation: int = 1, out: Optional[torch.Tensor] = None,
                             accumulate: bool = False, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
     """Eq. 4-5 retained term: dW[j,c,u,v] from dY [B,Cz,Ho,Wo] and the cache of a [B,Ca,H,W]; fp32."""
+    cache = dropit_dequantize_cache(cache)
     _require_cuda(dy, "dy")
     if dy.dtype != cache.dtype:
         raise TypeError("dy dtype %s != cache dtype %s" % (dy.dtype, cache.dtype))

@@ -48,7 +48,7 @@ class DropITLinearFn(torch.autograd.Function):
     """y = x W^T + b with the cached x replaced by its min-k compression."""
 
     @staticmethod
-    def forward(ctx, x, weight, bias, gamma: float, fmt: str, seed=None):
+    def forward(ctx, x, weight, bias, gamma: float, fmt: str, seed=None, quant: bool = False):
         _check_input(x)
         z = F.linear(x, weight, bias)
         ctx.has_bias = bias is not None
@@ -63,7 +63,12 @@ class DropITLinearFn(torch.autograd.Function):
                 x2 = x2.contiguous()
             cache = _compress(x2, gamma, fmt, seed)
             ctx.cache_meta = (cache.n, cache.k, cache.shape, cache.dtype, cache.fmt, cache.gamma)
-            ctx.save_for_backward(weight, cache.values, cache.meta, cache.offsets)
+            ctx.quant = bool(quant) and cache.dtype == torch.bfloat16
+            if ctx.quant:   # the retained values as 8-bit codes: 1 byte per retained element
+                cache = api.dropit_quantize_cache(cache)
+                ctx.save_for_backward(weight, cache.codes, cache.meta, cache.offsets, cache.scale)
+            else:
+                ctx.save_for_backward(weight, cache.values, cache.meta, cache.offsets)
         else:
             ctx.save_for_backward(weight)
         return z
@@ -78,14 +83,17 @@ class DropITLinearFn(torch.autograd.Function):
             dx = (dz2 @ weight.to(dz2.dtype)).reshape(ctx.x_shape).to(ctx.x_dtype)   # Eq. 3: exact, needs theta only
         if ctx.needs_input_grad[1] and ctx.cache_meta is not None:
             n, k, shape, dtype, fmt, gamma = ctx.cache_meta
-            cache = api.DropITCache(saved[1], saved[2], saved[3], n, k, shape, dtype, fmt, gamma)
+            if ctx.quant:
+                cache = api.DropITCache(None, saved[2], saved[3], n, k, shape, dtype, fmt, gamma, saved[1], saved[4])
+            else:
+                cache = api.DropITCache(saved[1], saved[2], saved[3], n, k, shape, dtype, fmt, gamma)
             dzc = dz2 if dz2.is_contiguous() else dz2.contiguous()
             if dzc.dtype != dtype:
                 dzc = dzc.to(dtype)
             dw = api.dropit_weight_grad(dzc, cache).to(weight.dtype)   # Eq. 6
         if ctx.has_bias and ctx.needs_input_grad[2]:
             db = dz2.sum(0).to(ctx.bias_dtype)
-        return dx, dw, db, None, None, None
+        return dx, dw, db, None, None, None, None
 
 
 class DropITConv2dFn(torch.autograd.Function):
@@ -185,15 +193,16 @@ class DropITLinear(nn.Linear, _Strategy):
     """nn.Linear whose backward uses a compressed input cache. `gamma` is the dropped fraction."""
 
     def __init__(self, in_features, out_features, bias=True, gamma: float = 0.9, fmt: str = "bitmask",
-                 strategy: str = "min_k", seed: int = 0, **kw):
+                 strategy: str = "min_k", seed: int = 0, quantize: bool = False, **kw):
         super().__init__(in_features, out_features, bias=bias, **kw)
         self.gamma, self.fmt = float(gamma), fmt
+        self.quantize = bool(quantize)     # keep the retained values as 8-bit codes (bf16 activations only)
         self._init_strategy(strategy, seed)
 
     def forward(self, x):
         if not (self.training and torch.is_grad_enabled()):
             return F.linear(x, self.weight, self.bias)     # inference is unchanged (Sec. 3.5)
-        return DropITLinearFn.apply(x, self.weight, self.bias, self.gamma, self.fmt, self._next_seed())
+        return DropITLinearFn.apply(x, self.weight, self.bias, self.gamma, self.fmt, self._next_seed(), self.quantize)
 
 
 class DropITGeluLinear(nn.Linear):
