@@ -245,8 +245,6 @@ __device__ __forceinline__ void cluster_finish_chunks(uint32_t tmem_base, const 
                                                       int sub, int lane, int rank, int splits, int j0, int c0, int Ca,
                                                       int Cz, float* __restrict__ dw, int accumulate) {
     const int cpo = (kBN / 32) / splits;
-    const int pitch = cpo * 32 + 4;
-    const float* mine = reinterpret_cast<const float*>(xchg) + (size_t)(32 * g + lane) * pitch;
     const int rr0 = lane >> 3, q = lane & 7;
 #pragma unroll 1
     for (int cl = sub; cl < cpo; cl += kEpiSubs) {
@@ -263,10 +261,9 @@ __device__ __forceinline__ void cluster_finish_chunks(uint32_t tmem_base, const 
                 for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(r[e]);
             } else {
                 const int slot = s < rank ? s : s - 1;
-                const float* src = mine + (size_t)slot * kBM * pitch + cl * 32;
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
-                    const float4 v = *reinterpret_cast<const float4*>(src + e);
+                    const float4 v = *reinterpret_cast<const float4*>(xchg + xchg_offset(slot, cpo, cl, g, e / 4, lane));
                     acc[e] += v.x; acc[e + 1] += v.y; acc[e + 2] += v.z; acc[e + 3] += v.w;
                 }
             }
