@@ -31,7 +31,9 @@ dropit_status decompress_dispatch(const void* values, const void* meta, const ui
 // Plan
 // ---------------------------------------------------------------------------------------------
 constexpr int kStages = 4;
-constexpr int kEpiSubs = 1;                            // epilogue warps per TMEM lane quarter (more of them did not shorten the epilogue)
+constexpr int kPairBK = 128;                            // wg_pair_kernel: tokens per pipeline stage
+constexpr int kPairStages = 3;
+constexpr int kEpiSubs = 2;                            // epilogue warps per TMEM lane quarter
 constexpr int kEpiWarps = 4 * kEpiSubs;
 constexpr int kTcThreads = 64 + 32 * kEpiWarps;        // TMA warp, MMA warp, epilogue warps (idle until the accumulator is final)
 
@@ -39,6 +41,7 @@ struct WgPlan {
     bool tensor_core;
     bool fused;               // weight_grad_tmem.cu: the cache is expanded into tensor memory inside the GEMM (no dense scratch)
     bool cluster;             // the splits of a tile form a thread-block cluster and add up through shared memory
+    bool pair;                // CTA pairs compute 256 x 256 tiles (wg_pair_kernel); the splits add up through global memory
     int tiles_m, tiles_n, splits, kb_total, kb_per_split;
     size_t counters_off, counters_bytes;
     size_t dense_off, dense_bytes;
@@ -49,6 +52,13 @@ struct WgPlan {
 // The kernel without a scratch: bitmask caches whose rows are whole 128-element chunks.
 static bool fused_supported(int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format) {
     return dtype == DROPIT_BF16 && format == DROPIT_FMT_BITMASK && (Ca % DROPIT_CHUNK == 0) && (Cz % 8 == 0);
+}
+
+// DROPIT_WG_PATH picks a kernel where several apply (for comparisons): "fused" = no scratch, cache expanded into
+// tensor memory; "single" = dense scratch, one CTA per tile.  Default: dense scratch, CTA pairs.
+static bool wg_path_is(const char* name) {
+    const char* e = std::getenv("DROPIT_WG_PATH");
+    return e && std::strcmp(e, name) == 0;
 }
 
 static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format, bool fused) {
@@ -71,27 +81,30 @@ static WgPlan make_wg_plan(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype
         return p;
     }
     if (p.tensor_core) {
-        p.tiles_m = (int)((Cz + kBM - 1) / kBM);
+        p.pair = Cz > kBM && !wg_path_is("single");
+        p.tiles_m = p.pair ? 2 * (int)((Cz + 2 * kBM - 1) / (2 * kBM)) : (int)((Cz + kBM - 1) / kBM);
         p.tiles_n = (int)((Ca + kBN - 1) / kBN);
-        p.kb_total = (int)((M + kBK - 1) / kBK);
+        const int bk = p.pair ? kPairBK : kBK;
+        p.kb_total = (int)((M + bk - 1) / bk);
         const int tiles = p.tiles_m * p.tiles_n;
         int splits = sm_count() / tiles;
         if (splits < 1) splits = 1;
+        if (splits > 255) splits = 255;                                  // the tile counters hold eight bits
         if (splits > p.kb_total) splits = p.kb_total;
         p.kb_per_split = (p.kb_total + splits - 1) / splits;
         p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;   // every split owns >= 1 block
-        p.cluster = p.splits == 2 || p.splits == 4;
+        p.cluster = !p.pair && (p.splits == 2 || p.splits == 4);
     } else {
         p.tiles_m = (int)((Cz + 63) / 64);
         p.tiles_n = (int)((Ca + 63) / 64);
         p.splits = 1;
     }
     p.counters_off = 0;
-    p.counters_bytes = align_up((size_t)p.tiles_m * p.tiles_n * 8, 256);   // per tile: tickets drawn, partial planes published
+    p.counters_bytes = align_up((size_t)p.tiles_m * p.tiles_n * 64, 256);   // per tile and part: tickets drawn, shares published
     p.dense_off = p.counters_off + p.counters_bytes;
     p.dense_bytes = align_up((size_t)M * Ca * es, 256);
     p.partial_off = p.dense_off + p.dense_bytes;
-    p.partial_bytes = (p.splits > 1 && !p.cluster) ? align_up((size_t)p.splits * Cz * Ca * 4, 256) : 0;
+    p.partial_bytes = (p.splits > 1 && !p.cluster) ? (size_t)p.splits * p.tiles_m * p.tiles_n * kBM * kBN * 4 : 0;   // whole tiles
     p.total_bytes = p.partial_off + p.partial_bytes;
     if (p.total_bytes == 0) p.total_bytes = 256;
     return p;
@@ -116,27 +129,27 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols) {
+bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kBK};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// The same matrix seen as [cols / 64][rows][64]: one box {64, kBK, groups} brings `groups` adjacent 64-column
-// groups of kBK rows with a single copy, laid out group after group as the MN-major operand wants them.
+// The same matrix seen as [cols / 64][rows][64]: one box {64, box_rows, groups} brings `groups` adjacent 64-column
+// groups of box_rows rows with a single copy, laid out group after group as the MN-major operand wants them.
 // Needs cols % 64 == 0 (a partial last group would read past the end of a row).
-bool make_map_grouped_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int groups) {
+bool make_map_grouped_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int groups, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
     cuuint64_t strides[2] = {(cuuint64_t)cols * 2, 128};
-    cuuint32_t box[3] = {64, (cuuint32_t)kBK, (cuuint32_t)groups};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)groups};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -159,85 +172,168 @@ constexpr int kEpiWarpFloats = 32 * kEpiRowFloats;         // one warp's 32 x 32
 constexpr int kEpiSpinLimit = 1 << 20;
 constexpr size_t kTcSmemBytes = 1024 + (size_t)kStages * (kAStageBytes + kBStageBytes) + sizeof(TcSmem);
 
-// Epilogue of one 128 x 256 accumulator tile, run by the four warps that own the TMEM lane quarters.
-// Each 32 x 32 chunk goes TMEM -> registers -> shared memory (row pitch 36 floats) and leaves as full
-// 128-byte row segments.  A CTA that is not its tile's finisher stores the chunk into its split's
-// partial plane.  The finisher adds the planes in split order, taking its own term from the chunk, so
-// the sum does not depend on which split finishes last, and writes dW.
-__device__ __forceinline__ void epilogue_tile_staged(uint32_t tmem_base, float* stage, int g, int sub, int lane, int j0, int c0,
-                                                     int Ca, int Cz, int split, int splits, bool finisher,
-                                                     float* __restrict__ dw, int accumulate,
-                                                     float* __restrict__ partial) {
-    const size_t plane = (size_t)Cz * Ca;
+// Counters in a workspace that nobody initialises: a word holds (call number << 8) | count.  Every CTA that
+// will use a word first makes sure, early in the kernel, that it carries this call's number (a word that does
+// not is stale and is replaced by a zero count; if the replacement fails, another CTA of the tile has done it,
+// or has even counted already, which it only does on a fresh word).  After that the word is counted up with
+// plain atomic additions, one trip to L2 each.
+__device__ __forceinline__ void epoch_counter_freshen(uint32_t* word, uint32_t epoch) {
+    const uint32_t old = *reinterpret_cast<volatile uint32_t*>(word);
+    if ((old >> 8) != epoch) atomicCAS(word, old, epoch << 8);
+}
+__device__ __forceinline__ void freshen_tile_counters(uint32_t* tile_counters, uint32_t epoch, int t) {
+    if (t >= 0 && t < 2 * (kBN / 32)) epoch_counter_freshen(tile_counters + t, epoch);
+}
+
+// The split reduction through global memory, as the four epilogue warps of a CTA run it once their accumulator
+// is final (threads 64 .. 64 + 32 * kEpiWarps - 1; named barrier 1).  The tile's eight 32-column chunks form
+// 1, 2, 4 or 8 parts (as many as there are splits, rounded down to a power of two), each with its own ticket
+// counter, and the CTA of split s starts at part s % parts.  The last CTA to draw a part's ticket is that part's
+// finisher: it waits until the others have published their share of the part, adds the planes in split order
+// and writes dW; the others store their share into their plane and go on to the next part.  So every CTA of a
+// tile stores some parts and finishes others, and a CTA only ever waits for CTAs that are already running.
+constexpr int kMaxParts = kBN / 32;
+__device__ __forceinline__ void ticket_epilogue(uint32_t tmem_base, float* stage_base, int warp, int lane, int j0, int c0,
+                                                int Ca, int Cz, int split, int splits, float* __restrict__ dw,
+                                                int accumulate, float* __restrict__ partial, uint32_t* tickets,
+                                                uint32_t* done, uint32_t epoch, int* finisher_flag,
+                                                volatile int* abort_flag);
+
+// Chunks [ch_begin, ch_end) of one 128 x 256 accumulator tile, as the warp that owns TMEM lane quarter g runs
+// them.  A CTA that is not the part's finisher stores its chunks into its split's plane just as they come out
+// of tensor memory: planes are laid out [tile][chunk][lane quarter][4-column group (8)][lane (32)] float4, so a
+// store instruction of the warp is 512 contiguous bytes and the finisher's lane reads back exactly the columns
+// of its own row.  The finisher adds the planes in split order, taking its own term from tensor memory (the sum
+// does not depend on which split finishes), turns the chunk through shared memory (row pitch 36 floats) and
+// writes full 128-byte row segments of dW.
+constexpr int kPlaneTileFloats = kBM * kBN;
+__device__ __forceinline__ size_t plane_offset(int ch, int g, int e4, int lane) {
+    return (size_t)(((ch * 4 + g) * 8 + e4) * 32 + lane) * 4;
+}
+__device__ __forceinline__ void epilogue_chunks(uint32_t tmem_base, float* stage, int g, int sub, int lane, int j0, int c0,
+                                                int ch_begin, int ch_end, int Ca, int Cz, int split, int splits,
+                                                bool finisher, float* __restrict__ dw, int accumulate,
+                                                float* __restrict__ planes, size_t plane_stride) {
     const int rr0 = lane >> 3, q = lane & 7;
+    float4 ahead[8];
 #pragma unroll 1
-    for (int ch = sub; ch < kBN / 32; ch += kEpiSubs) {    // the warps of a lane quarter take every kEpiSubs-th chunk
+    for (int ch = ch_begin + sub; ch < ch_end; ch += kEpiSubs) {    // the warps of a lane quarter take every kEpiSubs-th chunk
+        uint32_t r[32];
+        if (!finisher) {
+            ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
+            ptx::tmem_ld_wait();
+            float* dst = planes + (size_t)split * plane_stride + plane_offset(ch, g, 0, lane);
+#pragma unroll
+            for (int e4 = 0; e4 < 8; ++e4)
+                __stcg(reinterpret_cast<float4*>(dst + e4 * 128),
+                       make_float4(__uint_as_float(r[4 * e4]), __uint_as_float(r[4 * e4 + 1]), __uint_as_float(r[4 * e4 + 2]),
+                                   __uint_as_float(r[4 * e4 + 3])));
+            continue;
+        }
+        float4 other[8];
+        if (splits == 2) {                       // the common case: the other plane's loads are one chunk ahead
+            if (ch == ch_begin + sub) {
+                const float* src = planes + (size_t)(1 - split) * plane_stride + plane_offset(ch, g, 0, lane);
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) other[e4] = __ldcg(reinterpret_cast<const float4*>(src + e4 * 128));
+            } else {
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) other[e4] = ahead[e4];
+            }
+            if (ch + kEpiSubs < ch_end) {
+                const float* src = planes + (size_t)(1 - split) * plane_stride + plane_offset(ch + kEpiSubs, g, 0, lane);
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) ahead[e4] = __ldcg(reinterpret_cast<const float4*>(src + e4 * 128));
+            }
+        }
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
+        ptx::tmem_ld_wait();
+        float acc[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+        for (int s = 0; s < splits; ++s) {       // fixed order over the splits
+            if (s == split) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(r[e]);
+            } else {
+                if (splits != 2) {
+                    const float* src = planes + (size_t)s * plane_stride + plane_offset(ch, g, 0, lane);
+#pragma unroll
+                    for (int e4 = 0; e4 < 8; ++e4) other[e4] = __ldcg(reinterpret_cast<const float4*>(src + e4 * 128));
+                }
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) {
+                    acc[4 * e4] += other[e4].x; acc[4 * e4 + 1] += other[e4].y;
+                    acc[4 * e4 + 2] += other[e4].z; acc[4 * e4 + 3] += other[e4].w;
+                }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<float4*>(stage + lane * kEpiRowFloats + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
+        __syncwarp();
         const int col = c0 + ch * 32 + 4 * q;
-        const bool col_ok = col < Ca;            // Ca is a multiple of 8
-        size_t off[8];
-        bool ok[8];
-        float4 acc[8];
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
             const int row = j0 + 32 * g + it * 4 + rr0;
-            ok[it] = col_ok && row < Cz;
-            off[it] = ok[it] ? (size_t)row * Ca + col : 0;
-            acc[it] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        if (finisher && accumulate) {
-#pragma unroll
-            for (int it = 0; it < 8; ++it)
-                if (ok[it]) acc[it] = *reinterpret_cast<const float4*>(dw + off[it]);
-        }
-        float4 other[8];
-        if (finisher && splits == 2) {           // the common case: the other plane's loads fly during the TMEM read
-#pragma unroll
-            for (int it = 0; it < 8; ++it)
-                other[it] = ok[it] ? __ldcg(reinterpret_cast<const float4*>(partial + (size_t)(1 - split) * plane + off[it]))
-                                   : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
-        ptx::tmem_ld_wait();
-#pragma unroll
-        for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<float4*>(stage + lane * kEpiRowFloats + e) =
-                make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
-                            __uint_as_float(r[e + 3]));
-        __syncwarp();
-        float4 own[8];
-#pragma unroll
-        for (int it = 0; it < 8; ++it)
-            own[it] = *reinterpret_cast<const float4*>(stage + (it * 4 + rr0) * kEpiRowFloats + 4 * q);
-        __syncwarp();
-        if (!finisher) {
-#pragma unroll
-            for (int it = 0; it < 8; ++it)
-                if (ok[it]) *reinterpret_cast<float4*>(partial + (size_t)split * plane + off[it]) = own[it];
-            continue;
-        }
-        for (int s = 0; s < splits; ++s) {       // fixed order over the splits
-            float4 v[8];
-            if (s == split) {
-#pragma unroll
-                for (int it = 0; it < 8; ++it) v[it] = own[it];
-            } else if (splits == 2) {
-#pragma unroll
-                for (int it = 0; it < 8; ++it) v[it] = other[it];
-            } else {
-#pragma unroll
-                for (int it = 0; it < 8; ++it)
-                    v[it] = ok[it] ? __ldcg(reinterpret_cast<const float4*>(partial + (size_t)s * plane + off[it]))
-                                   : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int it = 0; it < 8; ++it) {
-                acc[it].x += v[it].x; acc[it].y += v[it].y; acc[it].z += v[it].z; acc[it].w += v[it].w;
+            if (col < Ca && row < Cz) {          // Ca is a multiple of 8
+                float4 v = *reinterpret_cast<const float4*>(stage + (it * 4 + rr0) * kEpiRowFloats + 4 * q);
+                float* dst = dw + (size_t)row * Ca + col;
+                if (accumulate) {
+                    const float4 o = *reinterpret_cast<const float4*>(dst);
+                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                }
+                *reinterpret_cast<float4*>(dst) = v;
             }
         }
-#pragma unroll
-        for (int it = 0; it < 8; ++it)
-            if (ok[it]) *reinterpret_cast<float4*>(dw + off[it]) = acc[it];
+        __syncwarp();
+    }
+}
+
+__device__ __forceinline__ void ticket_epilogue(uint32_t tmem_base, float* stage_base, int warp, int lane, int j0, int c0,
+                                                int Ca, int Cz, int split, int splits, float* __restrict__ dw,
+                                                int accumulate, float* __restrict__ partial, uint32_t* tickets,
+                                                uint32_t* done, uint32_t epoch, int* finisher_flag,
+                                                volatile int* abort_flag) {
+    const int parts = splits >= 8 ? 8 : (splits >= 4 ? 4 : (splits >= 2 ? 2 : 1));
+    const int cpp = kMaxParts / parts;           // chunks per part
+    float* stage = stage_base + (warp - 2) * kEpiWarpFloats;
+    for (int pi = 0; pi < parts; ++pi) {
+        const int part = (split + pi) % parts;
+        if (splits > 1) {
+            if (threadIdx.x == 64) {
+                const uint32_t t = atomicAdd(tickets + part, 1u) & 0xFFu;
+                *finisher_flag = (t == (uint32_t)splits - 1) ? 1 : 0;
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+        }
+        const bool finisher = *finisher_flag != 0;
+        if (finisher && splits > 1) {
+            // the other splits of this tile have drawn this part's ticket, so they are running their epilogues
+            if (threadIdx.x == 64) {
+                const uint32_t want = (epoch << 8) | ((uint32_t)splits - 1);
+                int spins = 0;
+                while (*reinterpret_cast<volatile uint32_t*>(done + part) != want && !*abort_flag) {
+                    if (++spins > kEpiSpinLimit) { *abort_flag = 1; break; }
+                    __nanosleep(32);
+                }
+                __threadfence();
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+        }
+        if (!*abort_flag) {
+            ptx::tc_fence_after();
+            epilogue_chunks(tmem_base, stage, warp & 3, (warp - 2) >> 2, lane, j0, c0, part * cpp, (part + 1) * cpp, Ca, Cz, split,
+                            splits, finisher, dw, accumulate, partial + (size_t)blockIdx.x * kPlaneTileFloats,
+                            (size_t)gridDim.x * kPlaneTileFloats);
+        }
+        if (splits > 1) {
+            // publish this CTA's share of the part (also after an abort, so that the finisher's wait ends); the
+            // barrier also keeps thread 64 from redrawing finisher_flag while others still read it
+            if (!finisher) __threadfence();
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+            if (!finisher && threadIdx.x == 64) atomicAdd(done + part, 1u);
+        }
     }
 }
 
@@ -294,7 +390,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, int Ca, int Cz,
              int tiles_n, int splits, int kb_per_split, int kb_total, float* __restrict__ dw, int accumulate,
              float* __restrict__ partial, uint32_t* counters, int32_t* dev_status, int cluster_mode,
-             int grouped_maps, uint32_t wait_limit) {
+             int grouped_maps, uint32_t wait_limit, uint32_t epoch) {
     extern __shared__ uint8_t smem_raw[];
     // The dynamic window starts at the same offset in every CTA of the kernel, so this rounding gives
     // the same offsets in both CTAs of a cluster (the exchange below maps addresses between them).
@@ -394,43 +490,16 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
     } else {
         // ---------------- epilogue: TMEM -> global ----------------
         ptx::launch_dependents();   // a programmatically launched kernel behind this one may be brought up
+        if (!cluster_mode && splits > 1) freshen_tile_counters(counters + (size_t)tile * 2 * kMaxParts, epoch, (int)threadIdx.x - 64);
         bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, wait_limit);
         ok = __all_sync(kFullMask, ok) && !*abort_flag;
         if (!ok) *abort_flag = 1;
-        if (!cluster_mode) {
         // The accumulator is final, so every MMA has read its operands and every TMA copy has landed:
         // the pipeline buffers are free and serve as the staging area.
-        uint32_t* tickets = counters + tile;
-        uint32_t* done = counters + gridDim.x + tile;
-        if (splits > 1) {
-            if (threadIdx.x == 64) ctl->finisher = (atomicAdd(tickets, 1u) == (uint32_t)splits - 1) ? 1 : 0;
-            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
-        }
-        const bool finisher = ctl->finisher != 0;
-        if (finisher && splits > 1) {
-            // the other splits of this tile have drawn their tickets, so they are running their epilogues
-            if (threadIdx.x == 64) {
-                int spins = 0;
-                while (*reinterpret_cast<volatile uint32_t*>(done) < (uint32_t)splits - 1 && !*abort_flag) {
-                    if (++spins > kEpiSpinLimit) { *abort_flag = 1; break; }
-                    __nanosleep(64);
-                }
-                __threadfence();
-            }
-            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
-        }
-        if (!*abort_flag) {
-            ptx::tc_fence_after();
-            float* stage = reinterpret_cast<float*>(smem) + (warp - 2) * kEpiWarpFloats;
-            epilogue_tile_staged(tmem_base, stage, warp & 3, (warp - 2) >> 2, lane, j0, c0, Ca, Cz, split, splits, finisher, dw,
-                                 accumulate, partial);
-        }
-        if (!finisher) {   // publish the partial plane (also after an abort, so that the finisher's wait ends)
-            __threadfence();
-            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
-            if (threadIdx.x == 64) atomicAdd(done, 1u);
-        }
-        }   // ticket path
+        if (!cluster_mode)
+            ticket_epilogue(tmem_base, reinterpret_cast<float*>(smem), warp, lane, j0, c0, Ca, Cz, split, splits, dw,
+                            accumulate, partial, counters + (size_t)tile * 2 * kMaxParts, counters + (size_t)tile * 2 * kMaxParts + kMaxParts, epoch,
+                            &ctl->finisher, abort_flag);
     }
 
     if (cluster_mode) {
@@ -459,6 +528,232 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         if (*abort_flag) ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kBN);
+    }
+    if (*abort_flag && threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------------------------
+// tcgen05 kernel on CTA pairs: the two CTAs of a cluster (2, 1, 1) compute a 256 x 256 tile of dW with one
+// MMA stream.  Each CTA loads its own 128 rows of dY and only half of the 256 columns of x, so a token block
+// costs a CTA 32 KB of shared-memory traffic from L2 instead of 48 KB; that traffic, not the tensor cores,
+// bounds the single-CTA kernel above.  Each CTA ends up with its 128 x 256 accumulator in its own tensor
+// memory and runs the ticket epilogue on it (the splits of the token axis are separate clusters).
+//
+// Pipeline: both CTAs' producers point their copies at the full barrier of the even-ranked CTA (the leader), whose
+// producer announces the bytes of both; the leader's MMA thread waits there, issues the MMAs for both CTAs and
+// commits onto the empty barrier of both.  (Announcing from the other CTA as well, by an arrival sent through
+// the cluster, cost that producer more time per token block than the MMAs of the block take.)
+// A copy costs the TMA unit about 0.1 us whatever its size, on top of its bytes; with 64 tokens per stage that
+// fixed part alone came to more than the MMAs of a stage take, hence three deep stages of 128 tokens rather
+// than six of 64.  The slots are shared out among three producer threads in three warps (slot s belongs to
+// producer s % 3); two of them are epilogue warps, which have nothing else to do until the accumulator is final.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPairProducers = 3;
+static_assert(kPairStages % kPairProducers == 0, "every producer owns the same number of slots");
+constexpr int kPairAStageBytes = kBM * kPairBK * 2;
+constexpr int kPairBStageBytes = (kBN / 2) * kPairBK * 2;
+constexpr uint32_t kPairStageTx = kPairAStageBytes + kPairBStageBytes;
+struct PairSmem {
+    uint64_t full[kPairStages];
+    uint64_t empty[kPairStages];
+    uint64_t accum;
+    uint32_t tmem_base;
+    int abort_flag;
+    int finisher;
+    int consumed;                    // leader: token blocks whose operands the MMA thread has seen arrive
+    int issued[kPairStages];         // per slot: rounds this CTA's producers have issued
+    int peer_issued[kPairStages];    // leader: the other CTA's `issued`, stored by that CTA when its producers stop
+    int peer_abort;                  // leader: the other CTA gave up a wait
+};
+constexpr size_t kPairSmemBytes = 1024 + (size_t)kPairStages * (kPairAStageBytes + kPairBStageBytes) + sizeof(PairSmem);
+static_assert(kPairStages * (kPairAStageBytes + kPairBStageBytes) >= (int)(kEpiWarps * kEpiWarpFloats * sizeof(float)),
+              "the epilogue stages its chunks in the pipeline buffers");
+
+// One producer thread: token blocks i = p, p + 3, p + 6, ... of this CTA's range (block i lives in slot i % stages,
+// so the thread only ever touches the slots s with s % 3 == p).
+__device__ __forceinline__ void pair_producer(PairSmem* ctl, uint8_t* sA, uint8_t* sB, const CUtensorMap* map_dy,
+                                              const CUtensorMap* map_x, int p, int member, uint32_t leader_rank, int nkb,
+                                              int kb_begin, int j0, int cb, int grouped_maps, uint32_t wait_limit) {
+    volatile int* abort_flag = &ctl->abort_flag;
+    const uint32_t full0 = ptx::map_shared_to_cta(ptx::smem_u32(&ctl->full[0]), leader_rank);
+    int rounds[kPairStages / kPairProducers];
+#pragma unroll
+    for (int q = 0; q < kPairStages / kPairProducers; ++q) rounds[q] = 0;
+    bool go = true;
+    for (int base = 0; base < nkb && go; base += kPairStages) {
+        const uint32_t round_parity = (uint32_t)(base / kPairStages) & 1u;
+#pragma unroll
+        for (int q = 0; q < kPairStages / kPairProducers; ++q) {
+            const int s = p + q * kPairProducers;
+            const int i = base + s;
+            if (i >= nkb || !go) continue;
+            if (*abort_flag || (base > 0 && !ptx::mbar_wait_poll(&ctl->empty[s], round_parity ^ 1u, wait_limit))) {
+                *abort_flag = 1;
+                go = false;
+                continue;
+            }
+            const uint32_t bar = full0 + 8u * (uint32_t)s;
+            if (!member) ptx::mbar_arrive_expect_tx(&ctl->full[s], 2u * kPairStageTx);
+            const int k0 = (kb_begin + i) * kPairBK;
+            uint8_t* a = sA + s * kPairAStageBytes;
+            uint8_t* b = sB + s * kPairBStageBytes;
+            if (grouped_maps) {   // one copy per operand
+                ptx::tma_load_3d_pair(a, map_dy, 0, k0, j0 / 64, bar);
+                ptx::tma_load_3d_pair(b, map_x, 0, k0, cb / 64, bar);
+            } else {
+#pragma unroll
+                for (int g = 0; g < kBM / 64; ++g) ptx::tma_load_2d_pair(a + g * (64 * kPairBK * 2), map_dy, j0 + 64 * g, k0, bar);
+#pragma unroll
+                for (int g = 0; g < kBN / 128; ++g) ptx::tma_load_2d_pair(b + g * (64 * kPairBK * 2), map_x, cb + 64 * g, k0, bar);
+            }
+            rounds[q] += 1;
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < kPairStages / kPairProducers; ++q) {
+        const int s = p + q * kPairProducers;
+        ctl->issued[s] = rounds[q];
+        if (member) ptx::st_cluster_u32(ptx::map_shared_to_cta(ptx::smem_u32(&ctl->peer_issued[s]), leader_rank), (uint32_t)rounds[q]);
+    }
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+wg_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, int Ca, int Cz,
+               int tiles_n, int splits, int kb_per_split, int kb_total, float* __restrict__ dw, int accumulate,
+               float* __restrict__ partial, uint32_t* counters, int32_t* dev_status, int grouped_maps,
+               uint32_t wait_limit, uint32_t epoch) {
+    extern __shared__ uint8_t smem_raw[];
+    // same offsets in both CTAs: the MMA addresses the operands of both with one descriptor
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + kPairStages * kPairAStageBytes;
+    PairSmem* ctl = reinterpret_cast<PairSmem*>(sB + kPairStages * kPairBStageBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();
+    const int member = (int)(rank & 1u);           // 0: leader
+    const uint32_t leader_rank = rank & ~1u;
+    const int tile = blockIdx.x;                   // the pair's CTAs are neighbours along x
+    const int split = blockIdx.y;
+    const int pair = tile >> 1;
+    const int j0 = ((pair / tiles_n) * 2 + member) * kBM;
+    const int c0 = (pair % tiles_n) * kBN;
+    const int cb = c0 + member * (kBN / 2);        // the half of the tile's columns whose x this CTA loads
+    const int kb_begin = split * kb_per_split;
+    const int kb_end = min(kb_total, kb_begin + kb_per_split);
+    const int nkb = kb_end - kb_begin;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) {
+            ptx::mbar_init(&ctl->full[s], 1);
+            ptx::mbar_init(&ctl->empty[s], 1);
+            ctl->issued[s] = 0;
+            ctl->peer_issued[s] = 0;
+        }
+        ptx::mbar_init(&ctl->accum, 1);
+        ctl->abort_flag = 0;
+        ctl->finisher = 1;
+        ctl->consumed = 0;
+        ctl->peer_abort = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&map_dy);
+        ptx::prefetch_tensormap(&map_x);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(&ctl->tmem_base, kBN);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before();
+    ptx::cluster_sync_all();     // both CTAs' barriers exist before either CTA signals the other
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    volatile int* abort_flag = &ctl->abort_flag;
+
+    if (warp == 0) {
+        // ---------------- TMA producer 0 (both CTAs) ----------------
+        if (lane == 0) {
+            ptx::grid_dependency_wait();   // the dense scratch is written by the kernel before this one
+            pair_producer(ctl, sA, sB, &map_dy, &map_x, 0, member, leader_rank, nkb, kb_begin, j0, cb, grouped_maps, wait_limit);
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader only) ----------------
+        if (lane == 0 && member == 0) {
+            constexpr uint32_t idesc = ptx::make_idesc_bf16(2 * kBM, kBN, true, true);
+            constexpr uint32_t kGroupBytes = 64 * kPairBK * 2;   // one 64-wide M/N group: kPairBK rows of 128 bytes
+            const uint16_t both = (uint16_t)(3u << leader_rank);
+            int consumed = 0, s = 0;
+            uint32_t round_parity = 0;
+            for (int i = 0; i < nkb; ++i) {
+                if (*abort_flag || !ptx::mbar_wait_poll(&ctl->full[s], round_parity, wait_limit)) {
+                    *abort_flag = 1;
+                    break;
+                }
+                consumed = i + 1;
+                ptx::tc_fence_after();
+                const uint32_t a_addr = ptx::smem_u32(sA + s * kPairAStageBytes);
+                const uint32_t b_addr = ptx::smem_u32(sB + s * kPairBStageBytes);
+#pragma unroll
+                for (int kk = 0; kk < kPairBK / 16; ++kk) {
+                    const uint64_t ad = ptx::make_smem_desc_sw128(a_addr + kk * 2048, kGroupBytes, 1024);
+                    const uint64_t bd = ptx::make_smem_desc_sw128(b_addr + kk * 2048, kGroupBytes, 1024);
+                    ptx::umma_bf16_pair(tmem_base, ad, bd, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                }
+                ptx::umma_commit_pair(&ctl->empty[s], both);
+                if (++s == kPairStages) { s = 0; round_parity ^= 1u; }
+            }
+            ctl->consumed = consumed;
+            ptx::umma_commit_pair(&ctl->accum, both);   // also after an abort: tells both CTAs when the MMAs in flight are done
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> global (both CTAs, each its own 128 rows) ----------------
+        ptx::launch_dependents();
+        if (splits > 1) freshen_tile_counters(counters + (size_t)tile * 2 * kMaxParts, epoch, (int)threadIdx.x - 64);
+        if (warp - 2 >= 1 && warp - 2 < kPairProducers) {   // producers 1 and 2 first
+            if (lane == 0) {
+                ptx::grid_dependency_wait();
+                pair_producer(ctl, sA, sB, &map_dy, &map_x, warp - 2, member, leader_rank, nkb, kb_begin, j0, cb, grouped_maps, wait_limit);
+            }
+            __syncwarp();
+        }
+        bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, wait_limit);
+        ok = __all_sync(kFullMask, ok) && !*abort_flag;
+        if (!ok) *abort_flag = 1;
+        // every MMA has read its operands in both CTAs: the pipeline buffers serve as the staging area
+        ticket_epilogue(tmem_base, reinterpret_cast<float*>(smem), warp, lane, j0, c0, Ca, Cz, split, splits, dw, accumulate,
+                        partial, counters + (size_t)tile * 2 * kMaxParts, counters + (size_t)tile * 2 * kMaxParts + kMaxParts, epoch,
+                        &ctl->finisher, abort_flag);
+    }
+
+    // Neither CTA leaves while the other may still signal its barriers or read its shared memory.  After a wait
+    // was given up, copies may be in flight whose token block the MMA thread never took, and one CTA may have
+    // issued a block that the other did not: the leader squares the accounts of those barriers by hand (bytes that
+    // were announced but never sent are counted as arrived; bytes that were sent unannounced get their arrival)
+    // and waits for the rest, between two cluster barriers that keep the other CTA alive.
+    __syncthreads();
+    if (member && threadIdx.x == 0 && *abort_flag)
+        ptx::st_cluster_u32(ptx::map_shared_to_cta(ptx::smem_u32(&ctl->peer_abort), leader_rank), 1u);
+    ptx::cluster_sync_all();
+    if (!member && threadIdx.x == 0 && (*abort_flag || *reinterpret_cast<volatile int*>(&ctl->peer_abort))) {
+        *abort_flag = 1;
+        const int consumed = ctl->consumed;
+        for (int s = 0; s < kPairStages; ++s) {
+            const int taken = consumed > s ? (consumed - s + kPairStages - 1) / kPairStages : 0;   // rounds of slot s the MMAs took
+            const int mine = ctl->issued[s], theirs = *reinterpret_cast<volatile int*>(&ctl->peer_issued[s]);
+            if (mine <= taken && theirs <= taken) continue;
+            uint64_t* bar = &ctl->full[s];
+            if (mine <= taken) ptx::mbar_arrive_expect_tx(bar, kPairStageTx);     // only the other CTA's half is on its way
+            else if (theirs <= taken) ptx::mbar_complete_tx(bar, kPairStageTx);   // the other CTA's half never left
+            ptx::mbar_wait(bar, (uint32_t)taken & 1u, kWaitLimit);
+        }
+    }
+    ptx::tc_fence_before();
+    ptx::cluster_sync_all();
+    if (warp == 1) {
+        // tensor memory is given back by both CTAs, and only once no MMA can still write to it
+        ptx::mbar_wait_warp(&ctl->accum, 0, kWaitLimit);
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc_pair(tmem_base, kBN);
     }
     if (*abort_flag && threadIdx.x == 0 && dev_status) atomicExch(dev_status, (int)DROPIT_ERR_TIMEOUT);
 }
@@ -535,12 +830,7 @@ extern "C" dropit_status dropit_weight_grad_workspace(int64_t M, int64_t Ca, int
     return DROPIT_OK;
 }
 
-// DROPIT_WG_PATH=fused makes dropit_weight_grad take the kernel without a scratch wherever it applies
-// (for comparisons; the workspace that dropit_weight_grad_workspace states is then more than is used).
-static bool prefer_fused() {
-    const char* e = std::getenv("DROPIT_WG_PATH");
-    return e && std::strcmp(e, "fused") == 0;
-}
+static bool prefer_fused() { return wg_path_is("fused"); }
 
 static dropit_status weight_grad_impl(const void* dy, const void* values, const void* meta,
                                       const uint32_t* offsets, int64_t M, int64_t Ca, int64_t Cz, int64_t k,
@@ -586,20 +876,21 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
 
     CUtensorMap map_dy, map_x;
     const bool grouped = (Ca % 64 == 0) && (Cz % 64 == 0);
+    const int bk = plan.pair ? kPairBK : kBK;
     if (grouped) {
-        if (!make_map_grouped_bf16(&map_dy, dy, M, Cz, kBM / 64) || !make_map_grouped_bf16(&map_x, dense, M, Ca, kBN / 64))
+        if (!make_map_grouped_bf16(&map_dy, dy, M, Cz, kBM / 64, bk) ||
+            !make_map_grouped_bf16(&map_x, dense, M, Ca, (plan.pair ? kBN / 2 : kBN) / 64, bk))
             return DROPIT_ERR_CUDA;
-    } else if (!make_map_2d_bf16(&map_dy, dy, M, Cz) || !make_map_2d_bf16(&map_x, dense, M, Ca)) {
+    } else if (!make_map_2d_bf16(&map_dy, dy, M, Cz, bk) || !make_map_2d_bf16(&map_x, dense, M, Ca, bk)) {
         return DROPIT_ERR_CUDA;
     }
     uint32_t* counters = reinterpret_cast<uint32_t*>(ws + plan.counters_off);
     float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
-    if (plan.splits > 1 && !plan.cluster && cudaMemsetAsync(counters, 0, plan.counters_bytes, stream) != cudaSuccess)
-        return DROPIT_ERR_CUDA;
+    const uint32_t epoch = next_epoch() & 0xFFFFFFu;   // stamps the tile counters, which nobody zeroes
     static PerDeviceOnce smem_attr;
     if (smem_attr.needed()) {
-        if (cudaFuncSetAttribute(wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(wg_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes) != cudaSuccess)
             return DROPIT_ERR_CUDA;
         smem_attr.mark();
     }
@@ -607,27 +898,30 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(kTcThreads);
-    cfg.dynamicSmemBytes = kTcSmemBytes;
+    cfg.dynamicSmemBytes = plan.pair ? kPairSmemBytes : kTcSmemBytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     cfg.attrs = attr;
-    if (plan.cluster) {
+    if (plan.cluster || plan.pair) {
         attr[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
-        attr[cfg.numAttrs].val.clusterDim.x = 1;
-        attr[cfg.numAttrs].val.clusterDim.y = (unsigned)plan.splits;
+        attr[cfg.numAttrs].val.clusterDim.x = plan.pair ? 2u : 1u;
+        attr[cfg.numAttrs].val.clusterDim.y = plan.pair ? 1u : (unsigned)plan.splits;
         attr[cfg.numAttrs].val.clusterDim.z = 1;
         ++cfg.numAttrs;
     }
-    if (plan.splits == 1 || plan.cluster) {
-        // the kernel right before this one in the stream is the decompression (no counter memset in
-        // between): this kernel may be set up while that one drains; it waits before reading the scratch
-        attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
-        ++cfg.numAttrs;
-    }
-    if (cudaLaunchKernelEx(&cfg, wg_tc_kernel, map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n, plan.splits,
-                           plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status,
-                           plan.cluster ? 1 : 0, grouped ? 1 : 0, spin_limit(kWaitLimit)) != cudaSuccess) {
+    // the kernel right before this one in the stream is the decompression: this kernel may be set up while that
+    // one drains; it waits before reading the scratch
+    attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+    ++cfg.numAttrs;
+    const cudaError_t err =
+        plan.pair ? cudaLaunchKernelEx(&cfg, wg_pair_kernel, map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n, plan.splits,
+                                       plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status,
+                                       grouped ? 1 : 0, spin_limit(kWaitLimit), epoch)
+                  : cudaLaunchKernelEx(&cfg, wg_tc_kernel, map_dy, map_x, (int)Ca, (int)Cz, plan.tiles_n, plan.splits,
+                                       plan.kb_per_split, plan.kb_total, dw, accumulate, partial, counters, dev_status,
+                                       plan.cluster ? 1 : 0, grouped ? 1 : 0, spin_limit(kWaitLimit), epoch);
+    if (err != cudaSuccess) {
         (void)cudaGetLastError();
         return DROPIT_ERR_CUDA;
     }

@@ -15,8 +15,10 @@ constexpr int kAStageBytes = kBM * kBK * 2;
 constexpr int kBStageBytes = kBN * kBK * 2;
 constexpr uint32_t kWaitLimit = 1u << 22;
 
-// Row-major bf16 matrix [rows, cols]; box = 64 columns (128 bytes) x kBK rows, 128-byte swizzle.
-bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols);
+// Row-major bf16 matrix [rows, cols]; box = 64 columns (128 bytes) x box_rows rows, 128-byte swizzle.
+bool make_map_2d_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows);
+// The same matrix as [cols / 64][rows][64] (cols % 64 == 0): one box brings `groups` adjacent 64-column groups.
+bool make_map_grouped_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int groups, int box_rows);
 
 // cluster exchange, receive area: (splits - 1) slots x (256 / splits) columns x 128 rows of fp32; largest for 4 splits
 constexpr int kXchgMaxBytes = 3 * kBM * (kBN / 4) * 4;

@@ -451,7 +451,6 @@ wg_tmem_kernel(const __grid_constant__ CUtensorMap map_dy, const uint16_t* __res
 
 }  // namespace
 
-bool make_map_grouped_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int groups);
 
 // Tiles of 128 channels x 256 outputs; `splits` CTAs per tile along the token axis (1, 2 or 4: a cluster).
 dropit_status launch_wg_tmem(const void* dy, const void* values, const void* mask, const uint32_t* offsets, int64_t M,
@@ -459,7 +458,7 @@ dropit_status launch_wg_tmem(const void* dy, const void* values, const void* mas
                              int accumulate, int32_t* dev_status, cudaStream_t stream) {
     CUtensorMap map_dy;
     const bool grouped = (Cz % 64 == 0);
-    if (grouped ? !make_map_grouped_bf16(&map_dy, dy, M, Cz, kBN / 64) : !make_map_2d_bf16(&map_dy, dy, M, Cz))
+    if (grouped ? !make_map_grouped_bf16(&map_dy, dy, M, Cz, kBN / 64, kBK) : !make_map_2d_bf16(&map_dy, dy, M, Cz, kBK))
         return DROPIT_ERR_CUDA;
     static PerDeviceOnce attr;
     if (attr.needed()) {
