@@ -8,6 +8,7 @@ from __future__ import annotations
 import contextlib
 import ctypes
 import functools
+import os
 from dataclasses import dataclass
 from typing import Optional, Tuple
 
@@ -321,7 +322,7 @@ def _device_index(device) -> int:
 
 
 @functools.lru_cache(maxsize=4096)
-def _weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int, dev_index: int) -> int:
+def _weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int, dev_index: int, path: str) -> int:
     out = ctypes.c_size_t(0)
     with _on_device(torch.device("cuda", dev_index)):
         code = _lib.load().dropit_weight_grad_workspace(M, Ca, Cz, dtype, fmt, ctypes.byref(out))
@@ -330,8 +331,10 @@ def _weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int, dev_i
 
 
 def dropit_weight_grad_workspace(M: int, Ca: int, Cz: int, dtype: int, fmt: int, device=None) -> int:
-    """Scratch bytes of dropit_weight_grad on `device` (the plan depends on the device's SM count)."""
-    return _weight_grad_workspace(int(M), int(Ca), int(Cz), int(dtype), int(fmt), _device_index(device))
+    """Scratch bytes of dropit_weight_grad on `device` (the plan depends on the device's SM count, and on the
+    kernel that DROPIT_WG_PATH asks for, which the library reads at every call)."""
+    return _weight_grad_workspace(int(M), int(Ca), int(Cz), int(dtype), int(fmt), _device_index(device),
+                                  os.environ.get("DROPIT_WG_PATH", ""))
 
 
 def dropit_weight_grad(dy: torch.Tensor, cache: DropITCache, out: Optional[torch.Tensor] = None,

@@ -50,8 +50,7 @@ __device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, u
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
-// Bounded wait that polls without suspending the thread: for barriers whose arrivals come from the other CTA of a
-// pair (a suspended try_wait was seen to sleep through those for a long time).
+// Bounded wait that polls without suspending the thread (test_wait instead of try_wait).
 __device__ __forceinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, uint32_t limit) {
     for (uint32_t i = 0; i < limit; ++i) {
         uint32_t ok;

@@ -2,20 +2,24 @@
 //   dW[j, c] = sum_n dY[n, j] * R(a-hat)[n, c]        dY [M, Cz], a [M, Ca], dW [Cz, Ca]
 //
 // The reduction runs over the token axis n, which is the strided axis of both row-major
-// operands, so for the tensor cores both operands are "MN-major": A = dY^T tile (128 output rows j),
-// B = R(a-hat) tile (256 output columns c), K = 64 tokens per pipeline stage.
+// operands, so for the tensor cores both operands are "MN-major": A = dY^T tile (128 output rows j per CTA),
+// B = R(a-hat) tile (256 output columns c), K = a block of tokens per pipeline stage.
 //
-// bf16: tcgen05.mma (kind::f16, fp32 accumulators in TMEM).  Two kernels:
-//  * this file: the cache is first inflated to a dense scratch matrix by the decompression kernel (it mostly stays
-//    in L2), both operands arrive by TMA in the 128-byte-swizzled canonical layout; one warp issues TMA, one
-//    thread issues MMAs, four warps drain TMEM.  The GEMM is launched programmatically behind the decompression
-//    and sets itself up while that one drains.  This is the faster variant on every measured shape and what
-//    dropit_weight_grad takes.
+// bf16: tcgen05.mma (kind::f16, fp32 accumulators in TMEM).  Three kernels:
+//  * wg_pair_kernel (this file; what dropit_weight_grad takes when Cz > 128): the cache is first inflated to a
+//    dense scratch matrix by the decompression kernel (it mostly stays in L2); CTA pairs (cta_group::2) compute
+//    256 x 256 tiles, each CTA loading its 128 rows of dY and half of the 256 columns of the scratch by TMA in
+//    the 128-byte-swizzled canonical layout.  The kernel is bound by shared-memory bandwidth (every operand byte
+//    is written once by TMA and read once by the MMAs; the pair saves a third of the B traffic of one CTA alone).
+//    It is launched programmatically behind the decompression and sets itself up while that one drains.
+//  * wg_tc_kernel (this file; Cz <= 128, or DROPIT_WG_PATH=single): the same with one CTA per 128 x 256 tile.
 //  * weight_grad_tmem.cu (dropit_weight_grad_fused): no scratch; the cache is expanded into tensor memory in
 //    front of the MMAs.  One launch, no workspace, slower.
-// Small output matrices are split along n ("split-K").  2 or 4 splits of a tile form a thread-block cluster and
-// add up through distributed shared memory; other split counts store partial tiles and the last split to arrive
-// adds them in split order.  Either way the summation order is fixed.
+// Small output matrices are split along n ("split-K").  The splits of a tile add up through global memory:
+// the tile is cut into as many parts as there are splits, every CTA stores the parts it does not finish into its
+// plane of the workspace and finishes the others, tickets deciding who finishes what (wg_tc_kernel with 2 or 4
+// splits: the splits form a thread-block cluster and exchange through distributed shared memory instead).
+// Either way the summation order is fixed.
 // fp32 (and channel counts that are not a multiple of 8): an FFMA kernel with 64x64 tiles on the dense scratch.
 #include <cstdlib>
 #include <cstring>

@@ -25,15 +25,15 @@ SMALL = [
     di.small_linear(512, 256, 128, "bf16", 0.0),                       # gamma = 0: the dense gradient
     di.small_linear(512, 256, 128, "bf16", 1.0),                       # gamma = 1: zero gradient
     di.small_linear(8192, 256, 128, "bf16", 0.9),                      # one tile, deep split along tokens
-    di.small_linear(200, 2056, 1000, "bf16", 0.9),                     # 72 tiles x 2 splits: cluster of 2, ragged tiles
-    di.small_linear(512, 1792, 520, "bf16", 0.9),                      # 35 tiles x 4 splits: cluster of 4, ragged rows
+    di.small_linear(200, 2056, 1000, "bf16", 0.9),                     # 72 tiles x 2 splits, ragged tiles
+    di.small_linear(512, 1792, 520, "bf16", 0.9),                      # 35 tiles (42 in CTA pairs: a pair half past the last row), ragged rows
     # the scratch is produced inside the GEMM kernel (channel counts that are multiples of 64):
     di.small_linear(131, 192, 64, "bf16", 0.7),                        # ragged last step (n = 24 * 1024 + 576), ragged k-block
     di.small_linear(333, 320, 192, "bf16", 0.5),                       # two column tiles, the second one partial
     di.small_linear(700, 256, 256, "bf16", 0.2),                       # dense steps: more values than the look-ahead window
-    di.small_linear(4100, 1024, 1152, "bf16", 0.9),                    # 36 tiles x 4 splits: cluster of 4
-    di.small_linear(2000, 2048, 1152, "bf16", 0.8),                    # 72 tiles x 2 splits: cluster of 2
-    di.small_linear(1500, 1280, 384, "bf16", 0.9),                     # 15 tiles x 9 splits: partial planes + tickets
+    di.small_linear(4100, 1024, 1152, "bf16", 0.9),                    # 36 tiles (40 in CTA pairs) x 4 / 3 splits
+    di.small_linear(2000, 2048, 1152, "bf16", 0.8),                    # 72 tiles x 2 splits
+    di.small_linear(1500, 1280, 384, "bf16", 0.9),                     # 15 tiles x 9 splits (20 x 7 in CTA pairs): eight parts per tile
     di.small_linear(300, 256, 256, "bf16", 0.5),                       # half of every row retained: runs longer than the value window
     di.small_linear(777, 384, 200, "bf16", 0.6),                       # ragged tokens and outputs, dense rows
     di.small_linear(4096, 128, 8, "bf16", 0.95),                       # one channel tile, eight outputs
@@ -62,6 +62,19 @@ def test_weight_grad_matches_oracle(cuda_device, case, fmt):
     assert err <= TIGHT[case.dtype], err
     if case.gamma == 1.0:
         assert not got.any()
+
+
+# The kernel with one CTA per tile (taken for Cz <= 128, or on request): 2 or 4 splits add up inside a cluster,
+# other counts through global memory.
+ONE_CTA = [c for c in SMALL if c.dtype == "bf16" and c.Cz > 128 and c.Ca % 8 == 0 and c.Cz % 8 == 0 and c.M >= 200]
+
+
+@pytest.mark.parametrize("case", ONE_CTA, ids=lambda c: c.name)
+def test_weight_grad_one_cta_per_tile_matches_oracle(cuda_device, case, monkeypatch):
+    monkeypatch.setenv("DROPIT_WG_PATH", "single")
+    bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
+    ref = oracle.fc_weight_grad(dyb, bits, keep, case.M, case.Ca, case.Cz, dt)
+    assert max_rel_err(dw.cpu().numpy(), ref) <= TIGHT[case.dtype]
 
 
 FUSED = [c for c in SMALL if c.dtype == "bf16" and c.Ca % 128 == 0 and c.Cz % 8 == 0] + [
