@@ -186,10 +186,6 @@ int oracle_min_k(const void* x, int64_t n, double gamma, int dtype, uint8_t* kee
     return rc;
 }
 
-/* ---- encoders for a-hat = {a_Xr, X_r} (Sec. 3.2) ------------------------ */
-
-/* Occupancy bitmask: element i <-> bit (i mod 32) of 32-bit word (i div 32);
- * the unused high bits of the last word are 0.  words has ceil(n/32) entries. */
 /* D(.) with the random strategy (Sec. 3.3 "Random Elements"): the same number of elements is retained as
  * under min-k, chosen by rank instead of magnitude. */
 int oracle_random_k(int64_t n, double gamma, uint64_t seed, uint8_t* keep, int64_t* k_out) {
@@ -204,6 +200,10 @@ int oracle_random_k(int64_t n, double gamma, uint64_t seed, uint8_t* keep, int64
     return rc;
 }
 
+/* ---- encoders for a-hat = {a_Xr, X_r} (Sec. 3.2) ------------------------ */
+
+/* Occupancy bitmask: element i <-> bit (i mod 32) of 32-bit word (i div 32);
+ * the unused high bits of the last word are 0.  words has ceil(n/32) entries. */
 void oracle_encode_bitmask(const uint8_t* keep, int64_t n, uint32_t* words) {
     int64_t nw = (n + 31) / 32;
     for (int64_t w = 0; w < nw; ++w) words[w] = 0;

@@ -1,7 +1,8 @@
 // bf16 min-k selection + packing as ONE persistent cooperative kernel (Sec. 3.3 "Min-K Elements",
 // Sec. 3.2 a-hat = {a_Xr, X_r}).
 //
-// Every WARP owns one contiguous run of 512-element blocks and keeps it for the whole kernel, so
+// Every WARP owns one contiguous run of 1024-element super-blocks (two 512-element blocks) and keeps it for the
+// whole kernel, so
 // the ordered compaction needs no block-wide synchronisation and warps drift freely.
 //   sample  every CTA histograms the same 16 Ki-element jittered sample in shared memory and brackets
 //           the threshold key T between two keys [lo, hi] (6-sigma margin on the sample rank).
@@ -14,7 +15,7 @@
 //           histograms.  No second counting pass.
 //   phase 3 second read (L2 hits for tensors that fit L2): element i is retained iff key_i > T, or
 //           key_i == T and fewer than q equal keys precede it; #retained before i =
-//           gt_before + min(eq_before, q).  A lane owns 16 consecutive elements; retained values are
+//           gt_before + min(eq_before, q).  A lane owns 32 consecutive elements of a super-block; retained values are
 //           staged per warp and leave in aligned 16-byte pieces.
 // When the band is wider than the per-warp histogram (small tensors, which are not sampled; key
 // distributions that are flat around T; a sample that missed) a general path is taken instead:
@@ -179,20 +180,6 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
     return wprefix + inc - v;
 }
 
-// Optional phase timestamps of CTA 0 (build with -DDROPIT_PHASE_TIMING): FusedState::reserved holds
-// %globaltimer at each stamp.  Off in normal builds.
-#ifdef DROPIT_PHASE_TIMING
-__device__ __forceinline__ void phase_stamp(FusedState* st, int i) {
-    if (st != nullptr && blockIdx.x == 0 && threadIdx.x == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        reinterpret_cast<unsigned long long*>(st->reserved)[i] = t;
-    }
-}
-#else
-__device__ __forceinline__ void phase_stamp(FusedState*, int) {}
-#endif
-
 // ---------------------------------------------------------------------------------------------
 // Sample step: bracket the threshold key.  Every CTA runs it on the same 16 Ki elements (the first
 // CTA to ask brings them in from HBM, the others read them from L2) and therefore arrives at the
@@ -228,7 +215,6 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
         uint4* z = reinterpret_cast<uint4*>(bins);
         for (int i = threadIdx.x; i < kKeySpace / 8; i += kFusedThreads) z[i] = make_uint4(0, 0, 0, 0);
         __syncthreads();
-        phase_stamp(st, 8);
 #pragma unroll
         for (int r = 0; r < kSampleVecs / kFusedThreads; ++r) {
             uint32_t key[8];
@@ -237,7 +223,6 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
             for (int e = 0; e < 8; ++e) atomicAdd(&bins[key[e] >> 1], 1u << ((key[e] & 1u) * 16));
         }
         __syncthreads();
-        phase_stamp(st, 9);
         // ranks (counted from the largest key) that bracket the threshold with a 6-sigma margin
         const float S = (float)(kSampleVecs * 8);
         const float p = (float)((double)k / (double)n);
@@ -263,7 +248,6 @@ __device__ __forceinline__ void sample_band(const uint4* __restrict__ x, int64_t
         after_loads();   // what the caller wants in flight while the thresholds are worked out (issued earlier, it delays the sample)
         uint32_t total;
         const uint32_t excl = block_exclusive_scan(sum, s_warp, &total);
-        phase_stamp(st, 10);
         // key at descending rank r: cum_before < r <= cum_before + h
         if ((excl < R_hi && R_hi <= excl + sum) || (excl < R_lo && R_lo <= excl + sum)) {
             // one or two threads of the CTA get here: they read their counters again, in key order
@@ -497,7 +481,6 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     };
     uint32_t barrier_target = 0;
 
-    phase_stamp(st, 7);
     // the general path's totals start at zero; the grid barriers order this store before their first use
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         st->n_hi[0] = 0;
@@ -527,7 +510,6 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     uint32_t lo = sh.band[0], hi = sh.band[1];
     uint32_t T = 0, q = 0;
     uint32_t run_gt = 0, run_eq = 0;   // this warp's exclusive prefix (absolute)
-    phase_stamp(st, 0);
 
     for (int attempt = 0; attempt < 2; ++attempt) {
         if (attempt == 1) {
@@ -645,7 +627,6 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                 }
             }
             prefetched = false;
-            phase_stamp(st, 1);
             for (int o = 16; o > 0; o >>= 1) {
                 cnt_lo += __shfl_xor_sync(kFullMask, cnt_lo, o);
                 cnt_hi += __shfl_xor_sync(kFullMask, cnt_hi, o);
@@ -689,7 +670,6 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
                 return;
             }
         }
-        phase_stamp(st, 2);
         if (threadIdx.x == 0) sh.found = 0;
         // ---------------- phase 2: threshold key, tie quota, prefixes ----------------
         if (narrow) {
@@ -879,7 +859,6 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
         break;
     }
     __syncthreads();   // shared histograms are dead from here on; phase 3 reuses the memory
-    phase_stamp(st, 3);
 
     // ---------------- phase 3: ordered compaction, one warp per run of super-blocks ----------------
     // A lane owns 32 consecutive elements = one mask word, so a super-block costs one warp scan and the
@@ -1009,7 +988,6 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     }
     // the elements of the last, partial piece (the warp behind this one writes the rest of that piece)
     if (lane >= (int)foreign && head + lane < gpos) values[head + lane] = s_vals[lane];
-    phase_stamp(st, 5);
 }
 
 // ---------------------------------------------------------------------------------------------
