@@ -336,7 +336,17 @@ __device__ __forceinline__ void ticket_epilogue(uint32_t tmem_base, float* stage
             // barrier also keeps thread 64 from redrawing finisher_flag while others still read it
             if (!finisher) __threadfence();
             asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
-            if (!finisher && threadIdx.x == 64) atomicAdd(done + part, 1u);
+            if (threadIdx.x == 64) {
+                if (!finisher) {
+                    atomicAdd(done + part, 1u);
+                } else if (!*abort_flag) {
+                    // every other split has drawn its ticket and published: nobody touches the part's two words
+                    // again in this launch.  Zero is stale for every call number (numbers are never zero), so the
+                    // same launch replayed from a captured graph starts from a clean count as well.
+                    tickets[part] = 0u;
+                    done[part] = 0u;
+                }
+            }
         }
     }
 }
@@ -890,7 +900,8 @@ static dropit_status weight_grad_impl(const void* dy, const void* values, const 
     }
     uint32_t* counters = reinterpret_cast<uint32_t*>(ws + plan.counters_off);
     float* partial = reinterpret_cast<float*>(ws + plan.partial_off);
-    const uint32_t epoch = next_epoch() & 0xFFFFFFu;   // stamps the tile counters, which nobody zeroes
+    uint32_t epoch = next_epoch() & 0xFFFFFFu;   // stamps the tile counters, which nobody zeroes beforehand
+    if (epoch == 0) epoch = 1;                     // zero marks a word that a finished call left behind
     static PerDeviceOnce smem_attr;
     if (smem_attr.needed()) {
         if (cudaFuncSetAttribute(wg_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess ||
