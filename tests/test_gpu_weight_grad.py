@@ -170,6 +170,33 @@ def test_weight_grad_is_reproducible(cuda_device):
         assert torch.equal(dropit.dropit_weight_grad(dy, cache), dw)
 
 
+def test_weight_grad_replayed_from_a_captured_graph(cuda_device):
+    """The tile counters of the split reduction carry a number that the host draws per call; a captured launch
+    replays the same number, and still has to start from clean counts (the finisher of a part clears them)."""
+    case = di.small_linear(2000, 2048, 1152, "bf16", 0.8)      # two splits per tile
+    bits, dyb, dt, keep, cache, dw = _run(case, "bitmask", cuda_device)
+    dy = di.make_dy(case).to(cuda_device)
+    wb = dropit.dropit_weight_grad_workspace(case.M, case.Ca, case.Cz, 0, 0, cuda_device)
+    ws = torch.empty(wb, dtype=torch.uint8, device=cuda_device)
+    out = torch.empty_like(dw)
+    side = torch.cuda.Stream(device=cuda_device)
+    side.wait_stream(torch.cuda.current_stream(cuda_device))
+    with torch.cuda.stream(side):
+        dropit.dropit_weight_grad(dy, cache, out=out, workspace=ws)      # attributes and the status word exist before capture
+    torch.cuda.current_stream(cuda_device).wait_stream(side)
+    torch.cuda.synchronize(cuda_device)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        dropit.dropit_weight_grad(dy, cache, out=out, workspace=ws)
+    for _ in range(3):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize(cuda_device)
+        dropit.check_device_status(cuda_device)
+        assert torch.equal(out, dw)
+    assert torch.equal(dropit.dropit_weight_grad(dy, cache, workspace=ws), dw)   # an ordinary call on the same workspace
+
+
 FULL_SIZE = [di.VITB_FC1, di.VITB_FC2,
              di.with_gamma(di.VITDET_QKV, 0.5), di.with_gamma(di.VITDET_QKV, 0.8), di.VITDET_QKV,
              di.with_gamma(di.VITDET_FC1, 0.5), di.VITDET_FC1,
