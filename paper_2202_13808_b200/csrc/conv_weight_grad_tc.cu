@@ -200,6 +200,8 @@ struct ConvTcParams {
     int bnc, nv, vgroups;        // B tile = nv horizontal taps x bnc input channels (nv * bnc <= 256)
     int a_rows;                  // rows of dY the A copy brings (the rows of a 128-row tile that can exist)
     int gathered;                // strided filter: the scratch holds one pre-sampled copy per tap (u*S + v)
+    int flat_w;                  // > 0: planes are flattened into one row of H*W pixels and the vertical tap offset is
+                                 // flat_w pixels per filter row along that row (stride 1, output as large as the input)
     int tiles_c;
     int splits, kb_per_split, kb_total;
 };
@@ -270,6 +272,7 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
                 const int x0 = xblk * p.xb, y0 = yblk * p.yb;
                 tma_load_4d(sA + s * kAStageBytes, &maps.dy, x0, y0, j0, n, &ctl->full[s]);
                 if (p.gathered) tma_load_5d(sB + s * kBStageBytes, &maps.x, x0, y0, c0, n, u * p.S + v0, &ctl->full[s]);
+                else if (p.flat_w) tma_load_5d(sB + s * kBStageBytes, &maps.x, x0 + (u - p.pad) * p.flat_w, y0, c0, n, v0, &ctl->full[s]);
                 else tma_load_5d(sB + s * kBStageBytes, &maps.x, x0, y0 + u - p.pad, c0, n, v0, &ctl->full[s]);
                 issued = i + 1;
                 if (++xblk == p.nxb) {
@@ -372,6 +375,7 @@ struct ConvTcPlan {
     int H, W, Ho, Wo;          // geometry the kernel sees (a 1x1 filter flattens each plane into one row)
     int tiles;
     ConvTcParams p;
+    int row_w;                 // pixels per image row as the shifted copies are written (W of the caller's tensor)
     bool padded;               // the GEMM reads rewritten copies of X (rows not multiples of 8 pixels, or a strided filter)
     bool pad_dy;               // ... and a zero-padded copy of dY
     int copies;                // copies of X in the scratch: S (one per horizontal tap) or R*S (strided filter)
@@ -385,7 +389,18 @@ ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, 
     if (dtype != DROPIT_BF16 || S > kMaxTapsX || pad > kMaxTapsX - 1 || B < 1) return pl;
     int Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
     const bool gathered = stride != 1;
+    pl.row_w = W;
+    int flat_w = 0;
     if (!gathered && R == 1 && S == 1 && pad == 0) {   // plain GEMM over the flattened plane
+        W = H * W; H = 1; Wo = W; Ho = 1;
+    } else if (!gathered && Ho == H && Wo == W && (W & 7) == 0 && R <= 2 * pad + 1) {
+        // Output as large as the input, rows that are whole 16-byte groups: the planes of dY and of the shifted
+        // copies are flattened into rows of H*W pixels.  A k-block is 64 consecutive pixels of that row (no padding
+        // of short image rows, every tile row a whole aligned 128-byte line); filter row u reads the copy
+        // (u - pad) * W pixels further along, and what that puts before the first or after the last pixel of the
+        // plane (the image rows above and below) is outside the tensor map and arrives as zeros.  The horizontal
+        // taps are the shifted copies as before, whose rows are zero where the tap leaves the image row.
+        flat_w = W;
         W = H * W; H = 1; Wo = W; Ho = 1;
     }
     if (!gathered && Wo > W) return pl;
@@ -398,6 +413,7 @@ ConvTcPlan make_conv_tc_plan(int B, int Ca, int H, int W, int Cz, int R, int S, 
     ConvTcParams& p = pl.p;
     p.Ca = Ca; p.Cz = Cz; p.R = R; p.S = S; p.pad = pad;
     p.gathered = gathered ? 1 : 0;
+    p.flat_w = flat_w;
     // One k-block = 64 consecutive pixels of one image row, so a tile row is exactly one 128-byte
     // swizzle row.  (Boxes with a narrower inner extent and several image rows are not used: their
     // shared-memory footprint under the 128-byte swizzle is not the dense one.)
@@ -465,7 +481,7 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
             int64_t blocks = (groups + 255) / 256;
             if (blocks > (int64_t)sm_count() * 16) blocks = (int64_t)sm_count() * 16;
             shift_copies_kernel<<<(unsigned)blocks, 256, 0, stream>>>(reinterpret_cast<const uint4*>(dense0), dst, groups,
-                                                                     pl.W / 8);
+                                                                     (pl.p.flat_w ? pl.row_w : pl.W) / 8);
             st0 = check_launch();
             if (st0 != DROPIT_OK) return st0;
         }
