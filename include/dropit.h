@@ -21,6 +21,12 @@
  *    kernel stores DROPIT_ERR_TIMEOUT into *dev_status (if given), leaves its
  *    outputs undefined and returns normally.  dev_status is never cleared by
  *    the library.
+ *  - Workspaces need no initialisation.  The few words in them that synchronise
+ *    CTAs (a grid barrier, tile counters) are stamped with a number the host
+ *    draws per call and are left stale when the kernel ends, so a call may be
+ *    captured into a CUDA graph and replayed on the same workspace.  After a
+ *    launch that reported DROPIT_ERR_TIMEOUT those words may be left
+ *    mid-count: clear the workspace before replaying a graph on it.
  *  - gamma is the DROPPED fraction.  n is the number of elements of the layer
  *    input (every token / pixel / channel of the mini-batch counts: one global
  *    selection per layer call).  n must be < 2^31.

@@ -38,7 +38,7 @@ constexpr int kP1Blocks = 4 / kVpl;                            // blocks loaded 
 constexpr int kKeySpace = 1 << 15;
 constexpr int kWarpBins = 64;                                  // per-warp band histogram
 constexpr int kRowWords = kWarpBins + 2;                       // per-CTA row: bins, #key>hi, pad
-constexpr int kMaxGrid = 512;
+constexpr int kMaxGrid = 512;                                  // < 4096: departures are counted in 12 bits of the barrier word
 constexpr int kSampleVecs = 2048;                              // 16384 sampled elements
 constexpr int64_t kSampleMinElems = 1 << 19;                   // below this the band is the full key range
 constexpr int kBarrierSpinLimit = 1 << 22;
@@ -866,6 +866,8 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     // for global memory in aligned 16-byte pieces after every super-block; the < 8 that remain are
     // carried to the front of the buffer.
     ptx::launch_dependents();   // a programmatically launched kernel behind this one may be brought up
+    unsigned long long departed_before = 0;   // see the end of the kernel
+    if (barrier_target != 0 && threadIdx.x == 0) departed_before = atomicAdd(&st->barrier, 1ull << 20);
     const int64_t nwords = (n + 31) / 32;
     uint16_t* s_vals = s_vals_all + (size_t)warp * kStageVals;
     const uint32_t s_vals_addr = ptx_smem(s_vals);
@@ -988,6 +990,16 @@ fused_compress_kernel(const uint4* __restrict__ x, int64_t n, unsigned long long
     }
     // the elements of the last, partial piece (the warp behind this one writes the rest of that piece)
     if (lane >= (int)foreign && head + lane < gpos) values[head + lane] = s_vals[lane];
+    // Leave the barrier word stale.  A launch replayed from a captured graph carries the same epoch again; if the
+    // word still held this epoch with all arrivals, a CTA that reached the first barrier before CTA 0 has
+    // re-stamped the word would pass at once.  Every CTA that went through a barrier (the same ones in every CTA)
+    // counts its departure in bits 20..31 of the word, which no wait looks at and which only grow the value; the
+    // last one to leave stores zero, an epoch that no call carries.
+    // (The count was taken at the start of this phase, behind the last barrier, so that its trip to L2 is not on
+    // the kernel's tail.)
+    if (barrier_target != 0 && threadIdx.x == 0 &&
+        ((departed_before >> 20) & 0xFFFull) == (unsigned long long)gridDim.x - 1ull)
+        asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(&st->barrier), "l"(0ull) : "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1013,6 +1025,7 @@ dropit_status fused_compress_bf16_prepared(const void* x, int64_t n, int64_t k, 
     unsigned long long kk = (unsigned long long)k;
     int bpw = plan.blocks_per_warp;
     uint32_t epoch = next_epoch();
+    if (epoch == 0) epoch = 1;   // zero marks a barrier word that a finished call left behind
     size_t h0 = plan.hist_off[0], h1 = plan.hist_off[1], ao = plan.agg_off, ro = plan.rows_off;
     uint16_t* vals = reinterpret_cast<uint16_t*>(values);
     uint32_t* maskp = index32 ? nullptr : reinterpret_cast<uint32_t*>(meta);

@@ -144,6 +144,35 @@ def test_workspace_needs_no_initialisation(cuda_device):
     dropit.check_device_status(cuda_device)
 
 
+def test_compress_replayed_from_a_captured_graph(cuda_device):
+    """The grid barrier counts under a number that the host draws per call; a captured launch replays the same number
+    and must still start from a clean word (the last CTA to leave a launch clears it)."""
+    case = di.small_linear(700, 768, 1, "bf16", 0.9)      # sampled path: one grid barrier
+    x = di.make_x(case)
+    bits, dt, keep, k = oracle_cache(x, case.gamma)
+    xd = x.to(cuda_device)
+    nbytes = dropit.dropit_cache_sizes(case.n, case.gamma, dropit.BF16, dropit.FMT_BITMASK)[3]
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=cuda_device)
+    side = torch.cuda.Stream(device=cuda_device)
+    side.wait_stream(torch.cuda.current_stream(cuda_device))
+    with torch.cuda.stream(side):
+        dropit.dropit_compress(xd, case.gamma, "bitmask", workspace=ws)   # attributes and the status word exist before capture
+    torch.cuda.current_stream(cuda_device).wait_stream(side)
+    torch.cuda.synchronize(cuda_device)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        cache = dropit.dropit_compress(xd, case.gamma, "bitmask", workspace=ws)
+    for _ in range(4):
+        cache.values.zero_(); cache.meta.zero_(); cache.offsets.zero_()
+        graph.replay()
+        torch.cuda.synchronize(cuda_device)
+        dropit.check_device_status(cuda_device)
+        assert_cache_matches_oracle(cache, bits, dt, keep, k, "bitmask")
+    again = dropit.dropit_compress(xd, case.gamma, "bitmask", workspace=ws)      # an ordinary call on the same workspace
+    dropit.check_device_status(cuda_device)
+    assert_cache_matches_oracle(again, bits, dt, keep, k, "bitmask")
+
+
 def test_decompress_into_a_given_buffer(cuda_device):
     case = di.small_linear(300, 3072, 1, "bf16", 0.9, "gelu")
     x = di.make_x(case).to(cuda_device)
