@@ -522,17 +522,21 @@ def run_ours(args, rank, world, device):
     roof["gemm_kernel_estimate"] = {"decompress_ms": {"fc1": dec_ms[0], "fc2": dec_ms[1]},
                                     "gemm_ms": {"fc1": gemm_ms[0], "fc2": gemm_ms[1]}, "tflops": gemm_tfl,
                                     **fractions(gemm_tfl, "tensor", peaks)}
+    # headline = compulsory bytes (x read once + outputs) over the time of the call: the bytes that must cross HBM;
+    # the algorithmic rate (two reads of x, as a two-pass selection has; the second one is served by L2 on this
+    # 77.5 MB tensor) and the rate of the DRAM counters are reported beside it
     roof_c = {"kernel": "dropit_compress (one launch: sample, band histogram, threshold, ordered compaction)",
-              "bound": "hbm", "layer": LAYERS[1].name, "achieved": comp_gbs[1], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-              "bytes_per_call": comp_a[1], "avg_ms": comp_ms[1], "traffic": tr_c, "peak_source": peaks["source"],
-              "achieved_is": "algorithmic bytes (two reads of X + outputs) / time; the second read of this 77.5 MB "
-                             "tensor is served by L2, so the bytes that cross HBM are the compulsory ones",
-              "compulsory_gbs": comp_cgbs[1], "compulsory_frac": comp_cgbs[1] / peaks["hbm_gbs"],
+              "bound": "hbm", "layer": LAYERS[1].name, "achieved": comp_cgbs[1], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+              "achieved_is": "compulsory bytes (X once + values + mask + seek table) / time of the call, L2-cold inputs",
+              "bytes_per_call": comp_c[1], "avg_ms": comp_ms[1], "traffic": tr_c, "peak_source": peaks["source"],
+              "algorithmic_bytes_per_call": comp_a[1], "algorithmic_gbs": comp_gbs[1],
+              "algorithmic_frac": comp_gbs[1] / peaks["hbm_gbs"], "algorithmic_frac_of_nominal": comp_gbs[1] / NOMINAL["hbm_gbs"],
               "dram_gbs": tr_c / (comp_ms[1] * 1e-3) / 1e9 if tr_c else None,
-              "other_layer": {"layer": LAYERS[0].name, "achieved": comp_gbs[0], "frac": comp_gbs[0] / peaks["hbm_gbs"],
-                              "compulsory_gbs": comp_cgbs[0], "avg_ms": comp_ms[0],
+              "other_layer": {"layer": LAYERS[0].name, "achieved": comp_cgbs[0], "frac": comp_cgbs[0] / peaks["hbm_gbs"],
+                              "algorithmic_gbs": comp_gbs[0], "algorithmic_frac": comp_gbs[0] / peaks["hbm_gbs"],
+                              "avg_ms": comp_ms[0],
                               "note": "19.4 MB: fits L2, dominated by the kernel's fixed steps"}}
-    roof_c.update(fractions(comp_gbs[1], "hbm", peaks))
+    roof_c.update(fractions(comp_cgbs[1], "hbm", peaks))
     out = {
         "metric": METRIC, "value": value, "unit": "samples/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
