@@ -35,7 +35,7 @@ dropit_status decompress_dispatch(const void* values, const void* meta, const ui
 // Plan
 // ---------------------------------------------------------------------------------------------
 constexpr int kStages = 4;
-constexpr int kPairBK = 128;                            // wg_pair_kernel: tokens per pipeline stage
+constexpr int kPairBK = 144;                            // wg_pair_kernel: tokens per pipeline stage (three stages fill the shared memory)
 constexpr int kPairStages = 3;
 constexpr int kEpiSubs = 2;                            // epilogue warps per TMEM lane quarter
 constexpr int kEpiWarps = 4 * kEpiSubs;
@@ -558,7 +558,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
 // commits onto the empty barrier of both.  (Announcing from the other CTA as well, by an arrival sent through
 // the cluster, cost that producer more time per token block than the MMAs of the block take.)
 // A copy costs the TMA unit about 0.1 us whatever its size, on top of its bytes; with 64 tokens per stage that
-// fixed part alone came to more than the MMAs of a stage take, hence three deep stages of 128 tokens rather
+// fixed part alone came to more than the MMAs of a stage take, hence three deep stages of 144 tokens rather
 // than six of 64.  The slots are shared out among three producer threads in three warps (slot s belongs to
 // producer s % 3); two of them are epilogue warps, which have nothing else to do until the accumulator is final.
 // ---------------------------------------------------------------------------------------------
