@@ -177,20 +177,44 @@ gather_taps_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, 
     }
 }
 
-// dw[j,c,u,v] (=|+=) sum over splits of partial[split][tap][j][c]
-__global__ void __launch_bounds__(256)
+// dw[j,c,u,v] (=|+=) sum over splits of partial[split][tap][j][c].  A warp takes 32 consecutive outputs; the eight
+// warps of a block share out the splits (warp g adds splits g, g + 8, ... in ascending order, several loads in
+// flight), and the eight sums are added in warp order: a fixed order for a given split count.
+constexpr int kReduceGroups = 8;
+__global__ void __launch_bounds__(32 * kReduceGroups)
 conv_tc_reduce_kernel(const float* __restrict__ partial, int splits, int Cz, int Ca, int taps, float* __restrict__ dw,
                       int accumulate) {
+    __shared__ float sums[kReduceGroups][32];
     const int64_t plane = (int64_t)taps * Cz * Ca;
+    const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
     ptx::grid_dependency_wait();   // the partial tiles come from the kernel before this one
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < plane; i += (int64_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % Ca);
-        const int j = (int)((i / Ca) % Cz);
-        const int tap = (int)(i / ((int64_t)Ca * Cz));
+    for (int64_t base = (int64_t)blockIdx.x * 32; base < plane; base += (int64_t)gridDim.x * 32) {
+        const int64_t i = base + lane;
         float acc = 0.f;
-        for (int s = 0; s < splits; ++s) acc += __ldcg(partial + (int64_t)s * plane + i);
-        float* d = dw + ((int64_t)j * Ca + c) * taps + tap;
-        *d = accumulate ? (*d + acc) : acc;
+        if (i < plane) {
+            int s = g;
+            for (; s + 3 * kReduceGroups < splits; s += 4 * kReduceGroups) {
+                const float v0 = __ldcg(partial + (int64_t)s * plane + i);
+                const float v1 = __ldcg(partial + (int64_t)(s + kReduceGroups) * plane + i);
+                const float v2 = __ldcg(partial + (int64_t)(s + 2 * kReduceGroups) * plane + i);
+                const float v3 = __ldcg(partial + (int64_t)(s + 3 * kReduceGroups) * plane + i);
+                acc += v0; acc += v1; acc += v2; acc += v3;
+            }
+            for (; s < splits; s += kReduceGroups) acc += __ldcg(partial + (int64_t)s * plane + i);
+        }
+        sums[g][lane] = acc;
+        __syncthreads();
+        if (g == 0 && i < plane) {
+            float t = sums[0][lane];
+#pragma unroll
+            for (int w = 1; w < kReduceGroups; ++w) t += sums[w][lane];
+            const int c = (int)(i % Ca);
+            const int j = (int)((i / Ca) % Cz);
+            const int tap = (int)(i / ((int64_t)Ca * Cz));
+            float* d = dw + ((int64_t)j * Ca + c) * taps + tap;
+            *d = accumulate ? (*d + t) : t;
+        }
+        __syncthreads();
     }
 }
 
@@ -552,10 +576,10 @@ dropit_status conv_tc_run(const void* dy, const void* values, const void* meta, 
     st = check_launch();
     if (st != DROPIT_OK) return st;
     const int64_t count = (int64_t)R * S * Cz * Ca;
-    int64_t blocks = (count + 255) / 256;
+    int64_t blocks = (count + 31) / 32;
     if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
     cfg.gridDim = dim3((unsigned)blocks);
-    cfg.blockDim = dim3(256);
+    cfg.blockDim = dim3(32 * kReduceGroups);
     cfg.dynamicSmemBytes = 0;
     if (cudaLaunchKernelEx(&cfg, conv_tc_reduce_kernel, (const float*)partial, pl.p.splits, Cz, Ca, R * S, dw,
                            accumulate) != cudaSuccess) {
