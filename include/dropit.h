@@ -238,7 +238,12 @@ dropit_status dropit_compress_static(const void* x, int64_t n, double gamma, dro
 dropit_status dropit_decompress(const void* values, const void* meta, const uint32_t* offsets, int64_t n, int64_t k,
                                 dropit_dtype dtype, dropit_format format, void* x_dense_out, void* cuda_stream);
 
-/* Scratch bytes that dropit_weight_grad needs for these shapes. [host] */
+/* Scratch bytes that dropit_weight_grad needs for these shapes on the current device (the plan
+ * depends on its SM count): the dense scratch, 64 bytes of counters per output tile and, when the
+ * token axis is split, one fp32 plane of whole tiles per split.  The environment variable
+ * DROPIT_WG_PATH ("single": one CTA per tile instead of CTA pairs; "fused": the kernel of
+ * dropit_weight_grad_fused), read at every call, picks another kernel for comparisons and changes
+ * the figure; query and call under the same setting. [host] */
 dropit_status dropit_weight_grad_workspace(int64_t M, int64_t Ca, int64_t Cz, dropit_dtype dtype, dropit_format format,
                                            size_t* workspace_bytes);
 
@@ -260,7 +265,7 @@ dropit_status dropit_weight_grad(const void* dy, const void* values, const void*
 
 /*
  * Same result as dropit_weight_grad (Eq. 6), computed WITHOUT inflating the cache to a dense
- * scratch tensor: R(a-hat) (Sec. 3.2: recovery is a temporary) is rebuilt, 32 tokens x 32 channels
+ * scratch tensor: R(a-hat) (Sec. 3.2: recovery is a temporary) is rebuilt, 128 channels x 16 tokens
  * at a time, straight from mask words, seek-table entries and packed values, and stored into
  * tensor memory, where the tensor cores read it as an MMA operand.  One kernel launch, and the
  * workspace is not touched (it may be NULL / 0 bytes).  Needs dtype = DROPIT_BF16,
