@@ -197,10 +197,19 @@ __device__ __forceinline__ void freshen_tile_counters(uint32_t* tile_counters, u
 // and writes dW; the others store their share into their plane and go on to the next part.  So every CTA of a
 // tile stores some parts and finishes others, and a CTA only ever waits for CTAs that are already running.
 constexpr int kMaxParts = kBN / 32;
+__device__ __forceinline__ int ticket_parts(int splits) { return splits >= 8 ? 8 : (splits >= 4 ? 4 : (splits >= 2 ? 2 : 1)); }
+// Thread 64 draws the ticket of the part its CTA starts with as soon as the tile's counters are fresh, long before
+// the accumulator is final, so that the trip to L2 is not part of the epilogue.  (A ticket says "this split is
+// running", which is as true during the main loop as after it; the waits on the other side are bounded.)
+__device__ __forceinline__ uint32_t draw_first_ticket(uint32_t* tile_counters, int split, int splits) {
+    __syncwarp();   // threads 64..79 of this warp have just freshened the counters
+    if (threadIdx.x != 64 || splits <= 1) return 0u;
+    return atomicAdd(tile_counters + split % ticket_parts(splits), 1u) & 0xFFu;
+}
 __device__ __forceinline__ void ticket_epilogue(uint32_t tmem_base, float* stage_base, int warp, int lane, int j0, int c0,
                                                 int Ca, int Cz, int split, int splits, float* __restrict__ dw,
                                                 int accumulate, float* __restrict__ partial, uint32_t* tickets,
-                                                uint32_t* done, uint32_t epoch, int* finisher_flag,
+                                                uint32_t* done, uint32_t epoch, uint32_t first_ticket, int* finisher_flag,
                                                 volatile int* abort_flag);
 
 // Chunks [ch_begin, ch_end) of one 128 x 256 accumulator tile, as the warp that owns TMEM lane quarter g runs
@@ -297,16 +306,17 @@ __device__ __forceinline__ void epilogue_chunks(uint32_t tmem_base, float* stage
 __device__ __forceinline__ void ticket_epilogue(uint32_t tmem_base, float* stage_base, int warp, int lane, int j0, int c0,
                                                 int Ca, int Cz, int split, int splits, float* __restrict__ dw,
                                                 int accumulate, float* __restrict__ partial, uint32_t* tickets,
-                                                uint32_t* done, uint32_t epoch, int* finisher_flag,
+                                                uint32_t* done, uint32_t epoch, uint32_t first_ticket, int* finisher_flag,
                                                 volatile int* abort_flag) {
-    const int parts = splits >= 8 ? 8 : (splits >= 4 ? 4 : (splits >= 2 ? 2 : 1));
+    const int parts = ticket_parts(splits);
     const int cpp = kMaxParts / parts;           // chunks per part
     float* stage = stage_base + (warp - 2) * kEpiWarpFloats;
     for (int pi = 0; pi < parts; ++pi) {
         const int part = (split + pi) % parts;
         if (splits > 1) {
             if (threadIdx.x == 64) {
-                const uint32_t t = atomicAdd(tickets + part, 1u) & 0xFFu;
+                // the ticket of the first part was drawn when the kernel started (draw_first_ticket)
+                const uint32_t t = pi == 0 ? first_ticket : (atomicAdd(tickets + part, 1u) & 0xFFu);
                 *finisher_flag = (t == (uint32_t)splits - 1) ? 1 : 0;
             }
             asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
@@ -504,7 +514,11 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
     } else {
         // ---------------- epilogue: TMEM -> global ----------------
         ptx::launch_dependents();   // a programmatically launched kernel behind this one may be brought up
-        if (!cluster_mode && splits > 1) freshen_tile_counters(counters + (size_t)tile * 2 * kMaxParts, epoch, (int)threadIdx.x - 64);
+        uint32_t first_ticket = 0;
+        if (!cluster_mode && splits > 1) {
+            freshen_tile_counters(counters + (size_t)tile * 2 * kMaxParts, epoch, (int)threadIdx.x - 64);
+            if (warp == 2) first_ticket = draw_first_ticket(counters + (size_t)tile * 2 * kMaxParts, split, splits);
+        }
         bool ok = ptx::mbar_wait_warp(&ctl->accum, 0, wait_limit);
         ok = __all_sync(kFullMask, ok) && !*abort_flag;
         if (!ok) *abort_flag = 1;
@@ -513,7 +527,7 @@ wg_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
         if (!cluster_mode)
             ticket_epilogue(tmem_base, reinterpret_cast<float*>(smem), warp, lane, j0, c0, Ca, Cz, split, splits, dw,
                             accumulate, partial, counters + (size_t)tile * 2 * kMaxParts, counters + (size_t)tile * 2 * kMaxParts + kMaxParts, epoch,
-                            &ctl->finisher, abort_flag);
+                            first_ticket, &ctl->finisher, abort_flag);
     }
 
     if (cluster_mode) {
@@ -722,7 +736,11 @@ wg_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
     } else {
         // ---------------- epilogue: TMEM -> global (both CTAs, each its own 128 rows) ----------------
         ptx::launch_dependents();
-        if (splits > 1) freshen_tile_counters(counters + (size_t)tile * 2 * kMaxParts, epoch, (int)threadIdx.x - 64);
+        uint32_t first_ticket = 0;
+        if (splits > 1) {
+            freshen_tile_counters(counters + (size_t)tile * 2 * kMaxParts, epoch, (int)threadIdx.x - 64);
+            if (warp == 2) first_ticket = draw_first_ticket(counters + (size_t)tile * 2 * kMaxParts, split, splits);
+        }
         if (warp - 2 >= 1 && warp - 2 < kPairProducers) {   // producers 1 and 2 first
             if (lane == 0) {
                 ptx::grid_dependency_wait();
@@ -736,7 +754,7 @@ wg_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
         // every MMA has read its operands in both CTAs: the pipeline buffers serve as the staging area
         ticket_epilogue(tmem_base, reinterpret_cast<float*>(smem), warp, lane, j0, c0, Ca, Cz, split, splits, dw, accumulate,
                         partial, counters + (size_t)tile * 2 * kMaxParts, counters + (size_t)tile * 2 * kMaxParts + kMaxParts, epoch,
-                        &ctl->finisher, abort_flag);
+                        first_ticket, &ctl->finisher, abort_flag);
     }
 
     // Neither CTA leaves while the other may still signal its barriers or read its shared memory.  After a wait
