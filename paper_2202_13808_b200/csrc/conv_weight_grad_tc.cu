@@ -341,36 +341,50 @@ conv_wg_tc_kernel(const __grid_constant__ ConvMaps maps, const ConvTcParams p, f
             *abort_flag = 1;
         } else {
             ptx::tc_fence_after();
+            // Every MMA has read its operands: the pipeline buffers serve as a staging area.  A 32 x 32 chunk goes
+            // TMEM -> registers -> shared memory (row pitch 36 floats) and leaves as full 128-byte row segments
+            // (a lane storing its own row straight from registers writes 16 bytes every Ca * 4 bytes: 9 us per tile).
             const int g = warp & 3;
-            const int row = j0 + 32 * g + lane;
             const int taps = p.R * p.S;
             const bool vec_ok = (p.Ca & 3) == 0;
-            for (int ch = 0; ch * 32 < ncols; ++ch) {
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
-                ptx::tmem_ld_wait();
-                if (row < p.Cz) {
+            constexpr int kRowFloats = 36;
+            float* stage = reinterpret_cast<float*>(smem) + (warp - 2) * 32 * kRowFloats;
+            const int rr0 = lane >> 3, q = lane & 7;
+            if (j0 + 32 * g < p.Cz) {              // uniform over the warp: some of its rows exist
+                for (int ch = 0; ch * 32 < ncols; ++ch) {
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * g) << 16) + ch * 32, r);
+                    ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        const int col = ch * 32 + e;       // bnc is a multiple of 16: 4 columns share one tap
-                        if (col < ncols) {
-                            const int vi = col / p.bnc;
-                            const int c = c0 + (col - vi * p.bnc);
-                            const int tap = u * p.S + v0 + vi;
-                            float* dst = partial + (((size_t)split * taps + tap) * p.Cz + row) * p.Ca + c;
-                            if (vec_ok && c + 4 <= p.Ca) {
-                                *reinterpret_cast<float4*>(dst) =
-                                    make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]),
-                                                __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                            } else {
+                    for (int e = 0; e < 32; e += 4)
+                        *reinterpret_cast<float4*>(stage + lane * kRowFloats + e) =
+                            make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
+                                        __uint_as_float(r[e + 3]));
+                    __syncwarp();
+                    const int col = ch * 32 + 4 * q;   // bnc is a multiple of 16: 4 columns share one tap
+                    if (col < ncols) {
+                        const int vi = col / p.bnc;
+                        const int c = c0 + (col - vi * p.bnc);
+                        const int tap = u * p.S + v0 + vi;
 #pragma unroll
-                                for (int q = 0; q < 4; ++q)
-                                    if (c + q < p.Ca) dst[q] = __uint_as_float(r[e + q]);
+                        for (int it = 0; it < 8; ++it) {
+                            const int row = j0 + 32 * g + it * 4 + rr0;
+                            if (row < p.Cz) {
+                                const float4 v = *reinterpret_cast<const float4*>(stage + (it * 4 + rr0) * kRowFloats + 4 * q);
+                                float* dst = partial + (((size_t)split * taps + tap) * p.Cz + row) * p.Ca + c;
+                                if (vec_ok && c + 4 <= p.Ca) {
+                                    *reinterpret_cast<float4*>(dst) = v;
+                                } else {
+                                    if (c < p.Ca) dst[0] = v.x;
+                                    if (c + 1 < p.Ca) dst[1] = v.y;
+                                    if (c + 2 < p.Ca) dst[2] = v.z;
+                                    if (c + 3 < p.Ca) dst[3] = v.w;
+                                }
                             }
                         }
                     }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
         }
     } else {
